@@ -1,0 +1,115 @@
+"""ctypes front end of ``mage_oracle.c`` (fp64, by-definition; see the C file).
+
+TEST INFRASTRUCTURE ONLY: nothing in the product path may import this module.
+Every function takes float32 NumPy arrays whose values are bf16-exact and
+returns float64 / int32 NumPy arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "mage_oracle.c")
+_LIB = os.path.join(_HERE, "libmage_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (no fast-math, so fp64 sums keep their written order)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-std=c11", "-o", _LIB, _SRC, "-lm"])
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_topk.restype = ctypes.c_int
+        _lib.oracle_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def _f32(a):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return a, a.ctypes.data_as(ctypes.c_void_p)
+
+
+def exact_block_attn(Q, Kc, Vc, Kb, Vb, scale=None, return_lse=False):
+    """Exact attention of one block (Algorithm 1 main stream).  Q [H_q,B,d], Kc/Vc [H_kv,N,d], Kb/Vb [H_kv,B,d]."""
+    Q, pq = _f32(Q); Kc, pk = _f32(Kc); Vc, pv = _f32(Vc); Kb, pkb = _f32(Kb); Vb, pvb = _f32(Vb)
+    H_q, B, d = Q.shape
+    H_kv, N, _ = Kc.shape
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    O = np.empty((H_q, B, d), dtype=np.float64)
+    lse = np.empty((H_q, B), dtype=np.float64)
+    _load().oracle_exact_block_attn(pq, pk, pv, pkb, pvb, H_q, H_kv, B, d, ctypes.c_int64(N), ctypes.c_double(scale),
+                                    O.ctypes.data_as(ctypes.c_void_p), lse.ctypes.data_as(ctypes.c_void_p))
+    return (O, lse) if return_lse else O
+
+
+def block_score(Q, Kc, H_kv=None, scale=None):
+    """Per-block score of every prefix position (Eq. 4): [H_kv, N] float64, each row sums to 1."""
+    Q, pq = _f32(Q); Kc, pk = _f32(Kc)
+    H_q, B, d = Q.shape
+    H_kv, N, _ = Kc.shape
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    score = np.zeros((H_kv, N), dtype=np.float64)
+    _load().oracle_block_score(pq, pk, H_q, H_kv, B, d, ctypes.c_int64(N), ctypes.c_double(scale),
+                               score.ctypes.data_as(ctypes.c_void_p))
+    return score
+
+
+def topk(score, k):
+    """Top-k positions per KV head by full sort.  Returns (idx [H_kv,k] int32 ascending, -1 padded; k_eff)."""
+    score = np.ascontiguousarray(score, dtype=np.float64)
+    H_kv, N = score.shape
+    idx = np.empty((H_kv, k), dtype=np.int32)
+    k_eff = min(k, N)
+    for h in range(H_kv):
+        k_eff = _load().oracle_topk(score[h].ctypes.data_as(ctypes.c_void_p), ctypes.c_int64(N), int(k),
+                                    idx[h].ctypes.data_as(ctypes.c_void_p))
+    return idx, int(k_eff)
+
+
+def sparse_block_attn(Q, Kc, Vc, Kb, Vb, idx, k_eff, scale=None):
+    """Reuse step (Algorithm 1 Phase 2): attention over cache rows idx[h,:k_eff] plus the block's own keys."""
+    Q, pq = _f32(Q); Kc, pk = _f32(Kc); Vc, pv = _f32(Vc); Kb, pkb = _f32(Kb); Vb, pvb = _f32(Vb)
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    H_q, B, d = Q.shape
+    H_kv, N, _ = Kc.shape
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    O = np.empty((H_q, B, d), dtype=np.float64)
+    _load().oracle_sparse_block_attn(pq, pk, pv, pkb, pvb, idx.ctypes.data_as(ctypes.c_void_p), int(idx.shape[1]),
+                                     int(k_eff), H_q, H_kv, B, d, ctypes.c_int64(N), ctypes.c_double(scale),
+                                     O.ctypes.data_as(ctypes.c_void_p))
+    return O
+
+
+def recall(idx_ref, idx_other, k_eff):
+    """Eq. 3: |S(1) ∩ S(tau)| / k per KV head, from two [H_kv, k] index arrays."""
+    out = []
+    for a, b in zip(np.asarray(idx_ref), np.asarray(idx_other)):
+        out.append(len(set(a[:k_eff].tolist()) & set(b[:k_eff].tolist())) / max(1, k_eff))
+    return np.array(out)
+
+
+def run_block(q_steps, Kc, Vc, kb_steps, vb_steps, k, scale=None):
+    """One block of Algorithm 1 on one problem: Step 1 exact + score + top-k, then T-1 reuse steps.
+
+    q_steps [T,H_q,B,d], kb_steps/vb_steps [T,H_kv,B,d].  Returns dict with O_exact, score, idx, k_eff, O_sparse (list).
+    """
+    O1 = exact_block_attn(q_steps[0], Kc, Vc, kb_steps[0], vb_steps[0], scale)
+    sc = block_score(q_steps[0], Kc, scale=scale)
+    idx, k_eff = topk(sc, k)
+    Os = [sparse_block_attn(q_steps[t], Kc, Vc, kb_steps[t], vb_steps[t], idx, k_eff, scale)
+          for t in range(1, len(q_steps))]
+    return {"O_exact": O1, "score": sc, "idx": idx, "k_eff": k_eff, "O_sparse": Os}

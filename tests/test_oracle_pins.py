@@ -1,0 +1,196 @@
+"""Pins for the CPU oracle: it is checked against things other than itself.
+
+Brute force in NumPy on tiny inputs, library special cases (torch SDPA, torch.topk),
+a hand-derived worked example, closed forms and invariants (Algorithm 1, Eq. 2-4).
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from helpers import bf16_exact, brute_force_block, brute_force_sparse, brute_force_topk
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "worked_example.txt")
+
+
+def _rand_problem(rng, H_q, H_kv, B, N, d):
+    return (bf16_exact(rng, (H_q, B, d)), bf16_exact(rng, (H_kv, N, d)), bf16_exact(rng, (H_kv, N, d)),
+            bf16_exact(rng, (H_kv, B, d)), bf16_exact(rng, (H_kv, B, d)))
+
+
+@pytest.mark.parametrize("G", [1, 4, 7])
+@pytest.mark.parametrize("B,N,d", [(1, 5, 8), (4, 64, 16), (3, 37, 128)])
+def test_bruteforce_tiny(oracle_mod, G, B, N, d):
+    rng = np.random.default_rng(100 * G + B)
+    H_kv = 2
+    Q, Kc, Vc, Kb, Vb = _rand_problem(rng, G * H_kv, H_kv, B, N, d)
+    scale = 1.0 / np.sqrt(d)
+    O_ref, sc_ref = brute_force_block(Q, Kc, Vc, Kb, Vb, scale)
+    O = oracle_mod.exact_block_attn(Q, Kc, Vc, Kb, Vb)
+    sc = oracle_mod.block_score(Q, Kc)
+    np.testing.assert_allclose(O, O_ref, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(sc, sc_ref, rtol=1e-12, atol=1e-15)
+    for k in (1, 3, N, N + 4):
+        idx, k_eff = oracle_mod.topk(sc, k)
+        assert k_eff == min(k, N)
+        for h in range(H_kv):
+            np.testing.assert_array_equal(idx[h, :k_eff], brute_force_topk(sc_ref[h], k))
+            assert (idx[h, k_eff:] == -1).all()
+        Os = oracle_mod.sparse_block_attn(Q, Kc, Vc, Kb, Vb, idx, k_eff)
+        np.testing.assert_allclose(Os, brute_force_sparse(Q, Kc, Vc, Kb, Vb, idx, k_eff, scale), rtol=0, atol=1e-12)
+
+
+def test_worked_example(oracle_mod):
+    vals = {}
+    for line in open(GOLDEN):
+        if line.startswith("#") or not line.strip():
+            continue
+        key, *nums = line.split()
+        vals[key] = np.array([float(x) for x in nums])
+    ln = np.log
+    Q = np.array([[[1.0, 0.0]], [[0.0, 1.0]]], dtype=np.float32)             # [H_q=2, B=1, d=2]
+    Kc = np.array([[[ln(3), 0.0], [0.0, ln(5)]]], dtype=np.float32)          # [1, 2, 2]
+    Kb = np.array([[[ln(2), ln(2)]]], dtype=np.float32)
+    Vc = np.array([[[1.0, 0.0], [0.0, 1.0]]], dtype=np.float32)
+    Vb = np.array([[[1.0, 1.0]]], dtype=np.float32)
+    O = oracle_mod.exact_block_attn(Q, Kc, Vc, Kb, Vb, scale=1.0)
+    np.testing.assert_allclose(O.ravel(), vals["O_exact"], atol=3e-7)           # fp32 rounding of ln(.) only
+    sc = oracle_mod.block_score(Q, Kc, scale=1.0)
+    np.testing.assert_allclose(sc.ravel(), vals["score"], atol=3e-7)
+    idx, k_eff = oracle_mod.topk(sc, 1)
+    assert idx[0, 0] == int(vals["top1"][0]) and k_eff == 1
+    Os = oracle_mod.sparse_block_attn(Q, Kc, Vc, Kb, Vb, idx, k_eff, scale=1.0)
+    np.testing.assert_allclose(Os.ravel(), vals["O_sparse"], atol=3e-7)
+
+
+def test_matches_torch_sdpa_and_topk(oracle_mod):
+    """Exact pass == SDPA over concat(cache, block) with KV heads repeated G times; sparse == SDPA on gathered rows."""
+    rng = np.random.default_rng(7)
+    H_q, H_kv, B, N, d = 8, 2, 8, 300, 64
+    G = H_q // H_kv
+    Q, Kc, Vc, Kb, Vb = _rand_problem(rng, H_q, H_kv, B, N, d)
+    t = lambda a: torch.from_numpy(a).double()
+    K_all = torch.cat([t(Kc), t(Kb)], dim=1).repeat_interleave(G, dim=0)
+    V_all = torch.cat([t(Vc), t(Vb)], dim=1).repeat_interleave(G, dim=0)
+    ref = torch.nn.functional.scaled_dot_product_attention(t(Q), K_all, V_all).numpy()
+    O, lse = oracle_mod.exact_block_attn(Q, Kc, Vc, Kb, Vb, return_lse=True)
+    np.testing.assert_allclose(O, ref, atol=1e-12)
+    S = torch.einsum("gqd,gnd->gqn", t(Q), t(Kc).repeat_interleave(G, dim=0)) / np.sqrt(d)
+    np.testing.assert_allclose(lse, torch.logsumexp(S, dim=-1).numpy(), atol=1e-12)
+    sc = oracle_mod.block_score(Q, Kc)
+    sc_ref = torch.softmax(S, dim=-1).reshape(H_kv, G * B, N).mean(dim=1).numpy()
+    np.testing.assert_allclose(sc, sc_ref, rtol=1e-12)
+    k = 40
+    idx, k_eff = oracle_mod.topk(sc, k)
+    for h in range(H_kv):
+        assert set(idx[h].tolist()) == set(torch.topk(torch.from_numpy(sc[h]), k).indices.tolist())
+        assert (np.diff(idx[h]) > 0).all()
+    Kg = torch.stack([t(Kc)[h][idx[h]] for h in range(H_kv)])
+    Vg = torch.stack([t(Vc)[h][idx[h]] for h in range(H_kv)])
+    ref_s = torch.nn.functional.scaled_dot_product_attention(
+        t(Q), torch.cat([Kg, t(Kb)], 1).repeat_interleave(G, 0), torch.cat([Vg, t(Vb)], 1).repeat_interleave(G, 0)).numpy()
+    np.testing.assert_allclose(oracle_mod.sparse_block_attn(Q, Kc, Vc, Kb, Vb, idx, k_eff), ref_s, atol=1e-12)
+
+
+def test_invariants(oracle_mod):
+    rng = np.random.default_rng(11)
+    H_q, H_kv, B, N, d = 14, 2, 5, 193, 32
+    Q, Kc, Vc, Kb, Vb = _rand_problem(rng, H_q, H_kv, B, N, d)
+    sc = oracle_mod.block_score(Q, Kc)
+    # every softmax row sums to one, so the mean over rows does too (pins the prefix-only domain and the 1/(GB))
+    np.testing.assert_allclose(sc.sum(axis=1), 1.0, rtol=1e-13)
+    assert (sc > 0).all()
+    # k = N: the sparse step is the exact pass
+    idx, k_eff = oracle_mod.topk(sc, N)
+    assert k_eff == N and (idx == np.arange(N)).all()
+    O = oracle_mod.exact_block_attn(Q, Kc, Vc, Kb, Vb)
+    np.testing.assert_allclose(oracle_mod.sparse_block_attn(Q, Kc, Vc, Kb, Vb, idx, N), O, atol=1e-13)
+    # k > N behaves as k = N, padded with -1
+    idx2, k_eff2 = oracle_mod.topk(sc, N + 7)
+    assert k_eff2 == N and (idx2[:, N:] == -1).all()
+    # permuting cache positions permutes the score, maps the top-k set, leaves O unchanged
+    perm = rng.permutation(N)
+    sc_p = oracle_mod.block_score(Q, Kc[:, perm])
+    np.testing.assert_allclose(sc_p, sc[:, perm], rtol=1e-12)
+    np.testing.assert_allclose(oracle_mod.exact_block_attn(Q, Kc[:, perm], Vc[:, perm], Kb, Vb), O, atol=1e-12)
+    k = 17
+    idx_k, _ = oracle_mod.topk(sc, k)
+    idx_kp, _ = oracle_mod.topk(sc_p, k)
+    for h in range(H_kv):
+        assert set(perm[idx_kp[h]].tolist()) == set(idx_k[h].tolist())
+    # the sparse step does not depend on the order of the index list
+    Os = oracle_mod.sparse_block_attn(Q, Kc, Vc, Kb, Vb, idx_k, k)
+    shuffled = np.stack([rng.permutation(row) for row in idx_k]).astype(np.int32)
+    np.testing.assert_allclose(oracle_mod.sparse_block_attn(Q, Kc, Vc, Kb, Vb, shuffled, k), Os, atol=1e-13)
+    # top-k set is a prefix of the full sort and holds at least as much mass as any other k-set
+    for h in range(H_kv):
+        np.testing.assert_array_equal(idx_k[h], brute_force_topk(sc[h], k))
+        other = rng.choice(N, size=k, replace=False)
+        assert sc[h][idx_k[h]].sum() >= sc[h][other].sum()
+    # splitting the prefix in chunks and merging (m, L, O) by log-sum-exp reproduces the one-shot result
+    cut = 80
+    _, lse_a = oracle_mod.exact_block_attn(Q, Kc[:, :cut], Vc[:, :cut], Kb, Vb, return_lse=True)
+    _, lse_b = oracle_mod.exact_block_attn(Q, Kc[:, cut:], Vc[:, cut:], Kb, Vb, return_lse=True)
+    _, lse = oracle_mod.exact_block_attn(Q, Kc, Vc, Kb, Vb, return_lse=True)
+    np.testing.assert_allclose(np.logaddexp(lse_a, lse_b), lse, rtol=1e-13)
+
+
+def test_closed_forms(oracle_mod):
+    rng = np.random.default_rng(3)
+    H_q, H_kv, B, N, d = 4, 2, 3, 50, 16
+    Q, Kc, Vc, Kb, Vb = _rand_problem(rng, H_q, H_kv, B, N, d)
+    # all prefix keys equal: score is 1/N everywhere; with equal block keys too, O is the plain mean of all values
+    Kc_eq = np.broadcast_to(Kc[:, :1], Kc.shape).copy()
+    np.testing.assert_allclose(oracle_mod.block_score(Q, Kc_eq), 1.0 / N, rtol=1e-13)
+    Kb_eq = np.broadcast_to(Kc[:, :1], Kb.shape).copy()
+    O = oracle_mod.exact_block_attn(Q, Kc_eq, Vc, Kb_eq, Vb)
+    mean_v = np.concatenate([Vc, Vb], axis=1).astype(np.float64).mean(axis=1)       # [H_kv, d]
+    np.testing.assert_allclose(O, np.repeat(mean_v, H_q // H_kv, axis=0)[:, None, :].repeat(B, 1), atol=1e-13)
+    # zero queries: uniform attention
+    np.testing.assert_allclose(oracle_mod.block_score(np.zeros_like(Q), Kc), 1.0 / N, rtol=1e-13)
+    # one key far above the rest: its score tends to 1 and O to its value row
+    Qd = np.zeros_like(Q); Qd[..., 0] = 8.0
+    Kd = np.zeros_like(Kc); Kd[:, 7, 0] = 32.0                                      # logit 8*32/4 = 64 above the others
+    sc = oracle_mod.block_score(Qd, Kd)
+    assert np.all(sc[:, 7] >= 1 - 1e-15) and np.all(np.delete(sc, 7, axis=1) < 1e-25)
+    O = oracle_mod.exact_block_attn(Qd, Kd, Vc, np.zeros_like(Kb), Vb)
+    np.testing.assert_allclose(O, np.repeat(Vc[:, 7], H_q // H_kv, axis=0)[:, None, :].repeat(B, 1), atol=1e-20)
+    # B = G = 1: single-query decode attention; the score is the softmax row itself
+    q1, k1 = Q[:1, :1], Kc[:1]
+    s = (k1[0].astype(np.float64) @ q1[0, 0].astype(np.float64)) / np.sqrt(d)
+    p = np.exp(s - s.max()); p /= p.sum()
+    np.testing.assert_allclose(oracle_mod.block_score(q1, k1)[0], p, rtol=1e-13)
+    # N = 0: attention inside the block only
+    O0 = oracle_mod.exact_block_attn(Q, Kc[:, :0], Vc[:, :0], Kb, Vb)
+    ref0, _ = brute_force_block(Q, Kc[:, :0], Vc[:, :0], Kb, Vb, 1 / np.sqrt(d))
+    np.testing.assert_allclose(O0, ref0, atol=1e-13)
+    idx0, k0 = oracle_mod.topk(np.zeros((H_kv, 0)), 4)
+    assert k0 == 0 and (idx0 == -1).all()
+
+
+def test_ties_prefer_smaller_position(oracle_mod):
+    sc = np.array([[0.1, 0.3, 0.3, 0.1, 0.3, 0.05]])
+    idx, _ = oracle_mod.topk(sc, 2)
+    assert idx.tolist() == [[1, 2]]
+    idx, _ = oracle_mod.topk(sc, 4)
+    assert idx.tolist() == [[0, 1, 2, 4]]
+
+
+def test_recall_and_planted_structure(oracle_mod):
+    """Eq. 3 on the synthetic recipe: heavy positions are over-represented in the Step-1 set, drift keeps recall high."""
+    import dataclasses
+    from paper_2602_14209_b200 import workloads as W
+    w = dataclasses.replace(W.CONFIGS["cfg1_small"], N=1024, T=3)
+    pr = W.make_problem(w, 0)
+    f = lambda a: a.float().numpy()
+    sc1 = oracle_mod.block_score(f(pr["q"][0]), f(pr["kc"]))
+    idx1, k_eff = oracle_mod.topk(sc1, w.k)
+    for h in range(w.H_kv):
+        frac = len(set(idx1[h].tolist()) & set(pr["heavy"][h].tolist())) / w.n_heavy
+        assert frac > 0.9                          # chance level would be k/N = 0.25
+    for t in (1, 2):
+        idx_t, _ = oracle_mod.topk(oracle_mod.block_score(f(pr["q"][t]), f(pr["kc"])), w.k)
+        r = oracle_mod.recall(idx1, idx_t, k_eff)
+        assert ((r > 0.3) & (r <= 1.0)).all()
+    assert (oracle_mod.recall(idx1, idx1, k_eff) == 1.0).all()
