@@ -1,0 +1,153 @@
+/*
+ * libmage -- the per-block sparse-attention hot path of MAGE ([MASK]-Guided
+ * Sparse Attention for block-diffusion LLMs) for NVIDIA B200 (sm_100a).
+ *
+ * Three stages, one entry point each (paper: Algorithm 1 and Section 4):
+ *
+ *   mage_exact_select       Step 1 of a block (Phase 1): exact attention of the
+ *                           all-[MASK] block over the whole prefix KV cache plus
+ *                           the block's own keys, and, in the same call, the
+ *                           per-block score of every prefix position (Eq. 4).
+ *   mage_topk               per-KV-head Top-k of those scores (Eq. 4 / Eq. 2),
+ *                           meant to be enqueued on a side ("select") stream.
+ *   mage_sparse_block_attn  steps 2..T (Phase 2): attention over the k selected
+ *                           cache rows plus the block's own keys, one softmax.
+ *
+ * Notation (paper, Section 3.1): H_q query heads, H_kv KV heads, G = H_q/H_kv
+ * query heads per KV head with group(h) = {hG .. hG+G-1}, B tokens per block,
+ * N prefix length, d head dimension, k budget.  A batch holds P independent
+ * problems (layers of one model, or sequences of a serving batch).
+ *
+ * Conventions
+ *   - Plain C ABI.  Every pointer argument except the mage_kv_t itself is DEVICE
+ *     memory owned by the caller; the library allocates nothing and keeps no
+ *     state between calls.  `stream` is a cudaStream_t passed as void*.
+ *   - All calls only enqueue work on `stream` and return.  The return value
+ *     covers host-detectable errors; nothing is launched when it is not MAGE_OK.
+ *   - Device-detectable problems (an index outside [0, N_p), a page id outside
+ *     [0, num_pages), a bounded wait that expired) set bits in *dev_status
+ *     (optional, may be NULL) and the offending access is skipped; a kernel
+ *     never traps.
+ *   - bf16 tensors are row-major with the head dimension contiguous; the score
+ *     and all accumulation are fp32.
+ */
+#ifndef MAGE_H_
+#define MAGE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MAGE_OK = 0,
+    MAGE_ERR_INVALID_ARG = -1,  /* null pointer, bad shape, k < 1, ...              */
+    MAGE_ERR_UNSUPPORTED = -2,  /* valid but not built: d != 128, B > 64, ...       */
+    MAGE_ERR_WORKSPACE = -3,    /* workspace smaller than mage_workspace_bytes()   */
+    MAGE_ERR_CUDA = -4          /* a CUDA call failed while enqueueing              */
+} mage_status;
+
+/* bits of *dev_status */
+#define MAGE_DEV_BAD_INDEX 1u   /* indices[] entry outside [0, N_p): row skipped    */
+#define MAGE_DEV_BAD_PAGE 2u    /* block_table entry outside [0, num_pages): skipped */
+#define MAGE_DEV_TIMEOUT 4u     /* an in-kernel bounded wait gave up                */
+
+/* mage_kv_t.flags */
+#define MAGE_FLAG_SIMT_KERNELS 1  /* use the portable CUDA-core kernels for every stage (slow; for cross-checks) */
+
+/*
+ * Prefix KV cache "C" of Algorithm 1 for a batch of P problems, read-only.
+ *
+ * Contiguous (page_size == 0): element (p, h, j, c) of K is
+ *     k_cache[p*stride_p + h*stride_h + j*stride_n + c]     (strides in elements, c < d contiguous)
+ * and likewise for V.  Strides must be multiples of 8 elements.
+ * Paged (page_size > 0): k_cache / v_cache are pools [num_pages][H_kv][page_size][d];
+ * logical position j of problem p lives in pool page block_table[p*max_pages + j/page_size],
+ * row j % page_size.  Strides are ignored.
+ * seq_lens[p] = N_p <= N_max is the prefix length of problem p (NULL: every N_p = N_max).
+ * N_p = 0 is legal.  Cache rows at positions >= N_p are never used as data.
+ */
+typedef struct mage_kv {
+    int32_t P, H_q, H_kv, d;      /* d must be 128; H_q % H_kv == 0                    */
+    int32_t B;                    /* 1..64 block tokens                                */
+    int32_t page_size;            /* 0 = contiguous, else tokens per page (power of two >= 16) */
+    const void *k_cache, *v_cache;
+    int64_t stride_p, stride_h, stride_n;
+    const int32_t *block_table;   /* device [P][max_pages], paged only                 */
+    int32_t max_pages, num_pages;
+    const int32_t *seq_lens;      /* device [P] or NULL                                */
+    int32_t N_max;                /* host-known bound on N_p; row stride of `scores`   */
+    int32_t flags;                /* MAGE_FLAG_*                                       */
+} mage_kv_t;
+
+/*
+ * Bytes of device workspace that any call on this cache description needs
+ * (host-only arithmetic, no CUDA call).  k_max is the largest budget that will
+ * be passed.  Returns 0 for an invalid description.  The workspace must be
+ * 256-byte aligned; its contents need not be preserved between calls, and two
+ * calls that may overlap on the GPU need separate workspaces.
+ */
+size_t mage_workspace_bytes(const mage_kv_t *kv, int32_t k_max);
+
+/*
+ * Step 1 of a block: exact attention + block score (Algorithm 1, Phase 1:
+ * main-stream "Attn(Q, K, V, C)" and select-stream "A = softmax(Q K^T / sqrt d)",
+ * "alpha = 1/(GB) sum_{g,q} A[g,q,:]"; Eq. 4).
+ *
+ *   q      [P][H_q][B][d]  bf16   queries of the all-[MASK] block
+ *   k_blk  [P][H_kv][B][d] bf16   the block's own keys  (attended densely, no mask, self included)
+ *   v_blk  [P][H_kv][B][d] bf16   the block's own values
+ *   out    [P][H_q][B][d]  bf16   softmax over the N_p prefix keys and the B block keys, times V
+ *   scores [P][H_kv][N_max] fp32  scores[p][h][j] = 1/(G*B) * sum over g in group(h), q of
+ *                                 softmax_j over the PREFIX keys of sm_scale * <q[g][q], K[h][j]>,
+ *                                 for j < N_p; entries j >= N_p are left untouched.
+ *   sm_scale  applied in fp32 to the accumulated dot product (1/sqrt(d) in the paper)
+ */
+mage_status mage_exact_select(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk,
+                              float sm_scale, void *out, float *scores, void *workspace, size_t workspace_bytes,
+                              uint32_t *dev_status, void *stream);
+
+/*
+ * Top-k selection per KV head (Algorithm 1, "S <- Top-k(alpha)"; Eq. 4).
+ *
+ *   scores   [P][H_kv][N_max] fp32, non-negative, no NaN
+ *   indices  [P][H_kv][k] int32   the k_eff = min(k, N_p) positions with the largest score, in
+ *                                 ascending position order; equal scores go to the smaller position;
+ *                                 slots >= k_eff are set to -1
+ *   k_eff    [P] int32            min(k, N_p)
+ * Exact (a radix select on the fp32 bit patterns), deterministic.  Needs no
+ * workspace (the arguments are kept for symmetry; they may be NULL / 0).
+ */
+mage_status mage_topk(const float *scores, const int32_t *seq_lens, int32_t P, int32_t H_kv, int32_t N_max,
+                      int32_t k, int32_t *indices, int32_t *k_eff, void *workspace, size_t workspace_bytes,
+                      void *stream);
+
+/*
+ * Reuse step, run at each of the T-1 remaining denoising steps (Algorithm 1,
+ * Phase 2, "SparseAttn(Q, K, V, C[S])").
+ *
+ *   q, k_blk, v_blk, out   as in mage_exact_select, holding the current step's tensors
+ *   indices [P][H_kv][k] int32, k_eff [P] int32   as written by mage_topk.  Any order is accepted;
+ *       a position listed twice is attended twice.  The same tensors serve every step of the block
+ *       (the selection is fixed at Step 1), so they must stay alive and unmodified until the last
+ *       reuse step has run.
+ * Each query attends to cache rows indices[p][h][0 .. k_eff[p]-1] of its KV head and to all B
+ * block keys, in one softmax.  With k_eff = N_p the result equals the exact pass.
+ */
+mage_status mage_sparse_block_attn(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk,
+                                   const int32_t *indices, const int32_t *k_eff, int32_t k, float sm_scale,
+                                   void *out, void *workspace, size_t workspace_bytes, uint32_t *dev_status,
+                                   void *stream);
+
+/* Static, human-readable name of a status code. */
+const char *mage_status_string(mage_status s);
+
+/* Number of kernels the library has launched in this process (for bookkeeping in benchmarks). */
+uint64_t mage_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MAGE_H_ */

@@ -1,0 +1,182 @@
+// Host side of libmage: argument validation, workspace planning and kernel launches behind the C ABI.
+#include <atomic>
+#include <cstdio>
+
+#include "common.cuh"
+#include "simt_kernels.cuh"
+#include "topk.cuh"
+
+namespace mage {
+
+static std::atomic<uint64_t> g_launches{0};
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static bool valid_kv(const mage_kv_t *kv, mage_status *why) {
+    auto fail = [&](mage_status s) { if (why) *why = s; return false; };
+    if (!kv) return fail(MAGE_ERR_INVALID_ARG);
+    if (kv->P < 1 || kv->H_q < 1 || kv->H_kv < 1 || kv->H_q % kv->H_kv != 0 || kv->B < 1 || kv->N_max < 0 || kv->d < 1)
+        return fail(MAGE_ERR_INVALID_ARG);
+    if (kv->d != kD || kv->B > 64) return fail(MAGE_ERR_UNSUPPORTED);
+    if (kv->N_max > 0 && (!kv->k_cache || !kv->v_cache)) return fail(MAGE_ERR_INVALID_ARG);
+    if (kv->page_size < 0) return fail(MAGE_ERR_INVALID_ARG);
+    if (kv->page_size == 0) {
+        if (kv->stride_n < kD || kv->stride_n % 8 || kv->stride_h % 8 || kv->stride_p % 8 || kv->stride_h < 0 || kv->stride_p < 0)
+            return fail(MAGE_ERR_INVALID_ARG);
+    } else {
+        if (kv->page_size < 16 || (kv->page_size & (kv->page_size - 1))) return fail(MAGE_ERR_UNSUPPORTED);
+        if (kv->N_max > 0 && (!kv->block_table || kv->num_pages < 1)) return fail(MAGE_ERR_INVALID_ARG);
+        if ((int64_t)kv->max_pages * kv->page_size < kv->N_max) return fail(MAGE_ERR_INVALID_ARG);
+    }
+    if ((int64_t)kv->P * kv->H_kv > 65535 * 16) return fail(MAGE_ERR_UNSUPPORTED);
+    return true;
+}
+
+static KvView make_view(const mage_kv_t *kv) {
+    KvView v;
+    v.k = static_cast<const __nv_bfloat16 *>(kv->k_cache);
+    v.v = static_cast<const __nv_bfloat16 *>(kv->v_cache);
+    v.stride_p = kv->stride_p; v.stride_h = kv->stride_h; v.stride_n = kv->stride_n;
+    v.block_table = kv->block_table; v.seq_lens = kv->seq_lens;
+    v.max_pages = kv->max_pages; v.num_pages = kv->num_pages; v.page_size = kv->page_size;
+    v.N_max = kv->N_max;
+    v.P = kv->P; v.H_q = kv->H_q; v.H_kv = kv->H_kv; v.B = kv->B; v.G = kv->H_q / kv->H_kv; v.M = v.G * kv->B;
+    return v;
+}
+
+// Split of the prefix for the exact pass: enough (head, chunk) items to fill the 148 SMs a few times over,
+// chunks of at least 1024 keys and a multiple of 128 keys.  Pure function of the description.
+static Plan make_plan(const mage_kv_t *kv) {
+    Plan pl;
+    pl.M = kv->H_q / kv->H_kv * kv->B;
+    pl.Mw = (int)align_up(pl.M, 128);
+    const int64_t heads = (int64_t)kv->P * kv->H_kv;
+    int64_t want = (592 + heads - 1) / heads;
+    const int64_t max_chunks = kv->N_max > 0 ? (kv->N_max + 1023) / 1024 : 1;
+    if (want > max_chunks) want = max_chunks;
+    if (want < 1) want = 1;
+    int64_t len = kv->N_max > 0 ? (kv->N_max + want - 1) / want : 128;
+    len = (int64_t)align_up((size_t)len, 128);
+    pl.chunk_len = (int)len;
+    pl.n_chunks = kv->N_max > 0 ? (int)((kv->N_max + len - 1) / len) : 0;
+    const size_t items = (size_t)heads * (pl.n_chunks + 1);
+    size_t off = 0;
+    pl.off_part_o = off;  off += items * pl.Mw * kD;
+    pl.off_part_ml = off; off += items * pl.Mw * 2;
+    pl.off_neg_lse = off; off += (size_t)heads * pl.Mw;
+    pl.total_bytes = align_up(off * sizeof(float), 256);
+    return pl;
+}
+
+static mage_status launch_check() {
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        std::fprintf(stderr, "libmage: kernel launch failed: %s\n", cudaGetErrorString(e));
+        return MAGE_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return MAGE_OK;
+}
+
+template <typename K>
+static mage_status opt_in_smem(K kernel, size_t bytes) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess ? MAGE_OK : MAGE_ERR_CUDA;
+}
+
+static mage_status exact_select_simt(const mage_kv_t *kv, const KvView &view, const Plan &plan, const __nv_bfloat16 *q,
+                                     const __nv_bfloat16 *k_blk, const __nv_bfloat16 *v_blk, float sm_scale,
+                                     __nv_bfloat16 *out, float *scores, float *ws, unsigned *dev_status, cudaStream_t st) {
+    using namespace simt;
+    const float scale_log2 = sm_scale * kLog2e;
+    auto kern = attn_kernel<Mode::kExactPartial>;
+    if (opt_in_smem(kern, kSmemBytes) != MAGE_OK || opt_in_smem(score_kernel, kSmemBytes) != MAGE_OK) return MAGE_ERR_CUDA;
+    const int row_tiles = (view.M + kRows - 1) / kRows;
+    dim3 grid(row_tiles, plan.n_chunks + 1, kv->P * kv->H_kv);
+    kern<<<grid, kThreads, kSmemBytes, st>>>(view, plan, q, k_blk, v_blk, nullptr, nullptr, 0, scale_log2, ws, nullptr, dev_status);
+    if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    const int rows_total = kv->P * kv->H_kv * view.M;
+    combine_kernel<<<(rows_total + 3) / 4, 128, 0, st>>>(view, plan, ws, out);
+    if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    if (kv->N_max > 0) {
+        dim3 sgrid((kv->N_max + kKeys - 1) / kKeys, 1, kv->P * kv->H_kv);
+        score_kernel<<<sgrid, kThreads, kSmemBytes, st>>>(view, plan, q, scale_log2, ws, scores, dev_status);
+        if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    }
+    return MAGE_OK;
+}
+
+static mage_status sparse_simt(const mage_kv_t *kv, const KvView &view, const Plan &plan, const __nv_bfloat16 *q,
+                               const __nv_bfloat16 *k_blk, const __nv_bfloat16 *v_blk, const int *indices,
+                               const int *k_eff, int k, float sm_scale, __nv_bfloat16 *out, unsigned *dev_status,
+                               cudaStream_t st) {
+    using namespace simt;
+    auto kern = attn_kernel<Mode::kSparseFinal>;
+    if (opt_in_smem(kern, kSmemBytes) != MAGE_OK) return MAGE_ERR_CUDA;
+    dim3 grid((view.M + kRows - 1) / kRows, 1, kv->P * kv->H_kv);
+    kern<<<grid, kThreads, kSmemBytes, st>>>(view, plan, q, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, nullptr, out, dev_status);
+    return launch_check();
+}
+
+}  // namespace mage
+
+using namespace mage;
+
+extern "C" {
+
+size_t mage_workspace_bytes(const mage_kv_t *kv, int32_t k_max) {
+    if (!valid_kv(kv, nullptr) || k_max < 1) return 0;
+    return make_plan(kv).total_bytes;
+}
+
+mage_status mage_exact_select(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk, float sm_scale,
+                              void *out, float *scores, void *workspace, size_t workspace_bytes, uint32_t *dev_status,
+                              void *stream) {
+    mage_status why = MAGE_OK;
+    if (!valid_kv(kv, &why)) return why;
+    if (!q || !k_blk || !v_blk || !out || !workspace || (kv->N_max > 0 && !scores)) return MAGE_ERR_INVALID_ARG;
+    if (!(sm_scale > 0.f) || (reinterpret_cast<uintptr_t>(workspace) & 255)) return MAGE_ERR_INVALID_ARG;
+    const Plan plan = make_plan(kv);
+    if (workspace_bytes < plan.total_bytes) return MAGE_ERR_WORKSPACE;
+    const KvView view = make_view(kv);
+    return exact_select_simt(kv, view, plan, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_blk),
+                             static_cast<const __nv_bfloat16 *>(v_blk), sm_scale, static_cast<__nv_bfloat16 *>(out), scores,
+                             static_cast<float *>(workspace), dev_status, static_cast<cudaStream_t>(stream));
+}
+
+mage_status mage_topk(const float *scores, const int32_t *seq_lens, int32_t P, int32_t H_kv, int32_t N_max, int32_t k,
+                      int32_t *indices, int32_t *k_eff, void *workspace, size_t workspace_bytes, void *stream) {
+    (void)workspace; (void)workspace_bytes;
+    if (P < 1 || H_kv < 1 || N_max < 0 || k < 1 || !indices || !k_eff || (N_max > 0 && !scores)) return MAGE_ERR_INVALID_ARG;
+    topk_kernel<<<P * H_kv, kTopkThreads, 0, static_cast<cudaStream_t>(stream)>>>(scores, seq_lens, H_kv, N_max, k, indices, k_eff);
+    return launch_check();
+}
+
+mage_status mage_sparse_block_attn(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk,
+                                   const int32_t *indices, const int32_t *k_eff, int32_t k, float sm_scale, void *out,
+                                   void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream) {
+    mage_status why = MAGE_OK;
+    if (!valid_kv(kv, &why)) return why;
+    if (!q || !k_blk || !v_blk || !out || !indices || !k_eff || k < 1) return MAGE_ERR_INVALID_ARG;
+    if (!(sm_scale > 0.f)) return MAGE_ERR_INVALID_ARG;
+    (void)workspace; (void)workspace_bytes;
+    const Plan plan = make_plan(kv);
+    const KvView view = make_view(kv);
+    return sparse_simt(kv, view, plan, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_blk),
+                       static_cast<const __nv_bfloat16 *>(v_blk), indices, k_eff, k, sm_scale, static_cast<__nv_bfloat16 *>(out),
+                       dev_status, static_cast<cudaStream_t>(stream));
+}
+
+const char *mage_status_string(mage_status s) {
+    switch (s) {
+        case MAGE_OK: return "MAGE_OK";
+        case MAGE_ERR_INVALID_ARG: return "MAGE_ERR_INVALID_ARG";
+        case MAGE_ERR_UNSUPPORTED: return "MAGE_ERR_UNSUPPORTED";
+        case MAGE_ERR_WORKSPACE: return "MAGE_ERR_WORKSPACE";
+        case MAGE_ERR_CUDA: return "MAGE_ERR_CUDA";
+    }
+    return "MAGE_ERR_UNKNOWN";
+}
+
+uint64_t mage_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

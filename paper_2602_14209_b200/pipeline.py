@@ -1,0 +1,73 @@
+"""Per-block call sequence of Algorithm 1 on two CUDA streams (buffers, streams, events; no arithmetic).
+
+Step 1 runs ``mage_exact_select`` on the main stream; ``mage_topk`` is enqueued on a
+dedicated select stream behind an event, so whatever the caller puts on the main
+stream next (the FFN in a model, other sequences' sparse steps in a serving
+batch) overlaps it; the main stream joins once before the first reuse step.
+"""
+from __future__ import annotations
+
+from typing import Optional, Sequence
+
+import torch
+
+from . import binding as mb
+
+
+class BlockAttention:
+    """Owns the outputs and scratch of one batch of problems and issues the three library calls."""
+
+    def __init__(self, kv: mb.KVCache, k: int, sm_scale: Optional[float] = None, select_stream: Optional[torch.cuda.Stream] = None):
+        self.kv, self.k = kv, int(k)
+        self.sm_scale = float(kv.d) ** -0.5 if sm_scale is None else float(sm_scale)
+        dev = kv.device
+        self.out = torch.empty(kv.P, kv.H_q, kv.B, kv.d, dtype=torch.bfloat16, device=dev)
+        self.scores = torch.zeros(kv.P, kv.H_kv, max(kv.N_max, 1), dtype=torch.float32, device=dev)
+        self.indices = torch.full((kv.P, kv.H_kv, self.k), -1, dtype=torch.int32, device=dev)
+        self.k_eff = torch.zeros(kv.P, dtype=torch.int32, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.workspace = kv.new_workspace(self.k)
+        self.select_stream = select_stream if select_stream is not None else torch.cuda.Stream(device=dev)
+        self._scores_ready = torch.cuda.Event()
+        self._indices_ready = torch.cuda.Event()
+
+    def exact_select(self, q, k_blk, v_blk, out=None, stream=None):
+        """Step 1 on ``stream`` (default: current): exact attention -> out, block scores -> self.scores."""
+        out = self.out if out is None else out
+        mb.mage_exact_select(self.kv, q, k_blk, v_blk, self.sm_scale, out, self.scores, self.workspace, self.status, stream)
+        return out
+
+    def select_async(self, main_stream=None):
+        """Top-k on the select stream, ordered after the scores written on ``main_stream``; does not block it."""
+        main = torch.cuda.current_stream() if main_stream is None else main_stream
+        self._scores_ready.record(main)
+        self.select_stream.wait_event(self._scores_ready)
+        mb.mage_topk(self.scores, self.kv.seq_lens, self.kv.P, self.kv.H_kv, max(self.kv.N_max, 0), self.k, self.indices,
+                     self.k_eff, stream=self.select_stream)
+        self._indices_ready.record(self.select_stream)
+
+    def join(self, main_stream=None):
+        """The single synchronisation at the end of Phase 1: the main stream waits for the index sets."""
+        main = torch.cuda.current_stream() if main_stream is None else main_stream
+        main.wait_event(self._indices_ready)
+
+    def sparse_step(self, q, k_blk, v_blk, out=None, stream=None):
+        """One reuse step (Phase 2) with the index sets fixed at Step 1."""
+        out = self.out if out is None else out
+        mb.mage_sparse_block_attn(self.kv, q, k_blk, v_blk, self.indices, self.k_eff, self.k, self.sm_scale, out,
+                                  self.workspace, self.status, stream)
+        return out
+
+    def run_block(self, q_steps: Sequence[torch.Tensor], kb_steps, vb_steps, outs: Optional[Sequence[torch.Tensor]] = None):
+        """One block: Step 1, asynchronous selection, join, then len(q_steps)-1 reuse steps.  Returns the outputs."""
+        T = len(q_steps)
+        res = []
+        o = self.exact_select(q_steps[0], kb_steps[0], vb_steps[0], None if outs is None else outs[0])
+        res.append(o)
+        if T > 1 or True:
+            self.select_async()
+        if T > 1:
+            self.join()
+        for t in range(1, T):
+            res.append(self.sparse_step(q_steps[t], kb_steps[t], vb_steps[t], None if outs is None else outs[t]))
+        return res

@@ -1,0 +1,101 @@
+"""Runs the CUDA path through the binding and compares it with the CPU oracle, problem by problem.
+
+Tolerances (written here once, used by every parity test):
+  attention outputs (bf16 in, fp32 accumulate, bf16 out): max-abs 1e-2, mean-abs 1e-3 against the fp64 oracle;
+  top-k: the GPU set may differ from the oracle's only in positions whose oracle score lies within 1e-5
+  relative of the oracle's k-th largest score; indices distinct, in range, ascending, -1 padded;
+  scores (diagnostic bound): 2e-5 relative.
+"""
+import math
+
+import numpy as np
+import torch
+
+from paper_2602_14209_b200 import binding as mb
+from paper_2602_14209_b200 import workloads as W
+from paper_2602_14209_b200.pipeline import BlockAttention
+
+O_MAX_ABS, O_MEAN_ABS, TOPK_BAND, SCORE_REL = 1e-2, 1e-3, 1e-5, 2e-5
+
+
+def run_gpu_block(batch, w, flags=0, paged=False, k=None, steps=None):
+    """One block of Algorithm 1 on the GPU for a batch drawn by workloads.make_batch(device='cuda')."""
+    k = w.k if k is None else k
+    T = batch["q"].shape[0] if steps is None else steps
+    extra = {}
+    if paged:
+        k_pool, v_pool, table, _ = W.to_paged(batch["kc"], batch["vc"], batch["seq_lens"].tolist(), w.page_size or 64, seed=w.seed)
+        kv = mb.KVCache(k_pool, v_pool, w.H_q, w.B, seq_lens=batch["seq_lens"], block_table=table, N_max=batch["N_max"], flags=flags)
+        extra = {"k_pool": k_pool, "v_pool": v_pool, "table": table}
+    else:
+        kv = mb.KVCache(batch["kc"], batch["vc"], w.H_q, w.B, seq_lens=batch["seq_lens"], flags=flags)
+    ba = BlockAttention(kv, k)
+    outs = [torch.full_like(ba.out, float("nan")) for _ in range(T)]
+    ba.scores.fill_(-1.0)                      # entries beyond N_p must stay untouched
+    launches0 = mb.launch_count()
+    ba.run_block([batch["q"][t] for t in range(T)], [batch["kb"][t] for t in range(T)], [batch["vb"][t] for t in range(T)], outs)
+    torch.cuda.synchronize()
+    return {"outs": [o.float().cpu().numpy() for o in outs], "scores": ba.scores.cpu().numpy(),
+            "indices": ba.indices.cpu().numpy(), "k_eff": ba.k_eff.cpu().numpy(), "status": int(ba.status.item()),
+            "launches": mb.launch_count() - launches0, "k": k, "ba": ba, **extra}
+
+
+def check_topk_band(score_ref, idx_gpu, k, N):
+    """Band rule on one KV head: score_ref [N] float64 (oracle), idx_gpu [k] int32."""
+    k_eff = min(k, N)
+    sel = idx_gpu[:k_eff]
+    assert (idx_gpu[k_eff:] == -1).all(), "slots beyond k_eff must be -1"
+    assert ((sel >= 0) & (sel < N)).all(), "index out of range"
+    assert (np.diff(sel) > 0).all(), "indices must be ascending and distinct"
+    if k_eff == N or k_eff == 0:
+        return 0
+    tau = np.partition(score_ref, N - k_eff)[N - k_eff]            # k-th largest
+    must = np.nonzero(score_ref > tau * (1 + TOPK_BAND))[0]
+    never = score_ref < tau * (1 - TOPK_BAND)
+    chosen = np.zeros(N, dtype=bool)
+    chosen[sel] = True
+    assert chosen[must].all(), f"missing {np.sum(~chosen[must])} entries clearly above the k-th score"
+    assert not (chosen & never).any(), f"selected {np.sum(chosen & never)} entries clearly below the k-th score"
+    ref_set = np.argsort(-score_ref, kind="stable")[:k_eff]
+    return k_eff - int(chosen[ref_set].sum())                      # positions that differ (all inside the band)
+
+
+def check_problem(oracle, batch, res, w, p, heads=None, check_scores=True, sparse_steps=None):
+    """Compare problem p of a GPU run with the oracle on the listed KV heads (default: all).  Returns diagnostics."""
+    G, B, k = w.G, w.B, res["k"]
+    N = int(batch["seq_lens"][p])
+    heads = range(w.H_kv) if heads is None else heads
+    T = len(res["outs"])
+    diag = {"o_max": 0.0, "o_mean": 0.0, "score_rel": 0.0, "band_swaps": 0, "sp_max": 0.0, "sp_mean": 0.0}
+    f = lambda t: t.float().cpu().numpy()
+    assert res["k_eff"][p] == min(k, N)
+    for h in heads:
+        qs = slice(h * G, (h + 1) * G)
+        Kc, Vc = f(batch["kc"][p, h:h + 1, :N]), f(batch["vc"][p, h:h + 1, :N])
+        O = oracle.exact_block_attn(f(batch["q"][0, p, qs]), Kc, Vc, f(batch["kb"][0, p, h:h + 1]), f(batch["vb"][0, p, h:h + 1]))
+        err = np.abs(res["outs"][0][p, qs] - O)
+        assert np.isfinite(res["outs"][0][p, qs]).all()
+        diag["o_max"], diag["o_mean"] = max(diag["o_max"], err.max()), max(diag["o_mean"], err.mean())
+        assert err.max() <= O_MAX_ABS and err.mean() <= O_MEAN_ABS, (p, h, err.max(), err.mean())
+        if N > 0:
+            sc = oracle.block_score(f(batch["q"][0, p, qs]), Kc)[0]
+            got = res["scores"][p, h, :N].astype(np.float64)
+            rel = np.max(np.abs(got - sc) / sc)
+            diag["score_rel"] = max(diag["score_rel"], rel)
+            if check_scores:
+                assert rel <= SCORE_REL, (p, h, rel)
+            assert (res["scores"][p, h, N:] == -1.0).all(), "scores beyond N_p were written"
+            diag["band_swaps"] += check_topk_band(sc, res["indices"][p, h], k, N)
+        else:
+            assert (res["indices"][p, h] == -1).all()
+        k_eff = int(res["k_eff"][p])
+        for t in (range(1, T) if sparse_steps is None else sparse_steps):
+            idx = res["indices"][p, h:h + 1]
+            Os = oracle.sparse_block_attn(f(batch["q"][t, p, qs]), Kc, Vc, f(batch["kb"][t, p, h:h + 1]),
+                                          f(batch["vb"][t, p, h:h + 1]), idx, k_eff)
+            e = np.abs(res["outs"][t][p, qs] - Os)
+            assert np.isfinite(res["outs"][t][p, qs]).all()
+            diag["sp_max"], diag["sp_mean"] = max(diag["sp_max"], e.max()), max(diag["sp_mean"], e.mean())
+            assert e.max() <= O_MAX_ABS and e.mean() <= O_MEAN_ABS, (p, h, t, e.max(), e.mean())
+    assert res["status"] == 0
+    return diag

@@ -1,0 +1,137 @@
+"""GPU-vs-oracle parity through the C ABI (binding -> libmage.so), element by element on seeded inputs."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+from paper_2602_14209_b200 import binding as mb
+from paper_2602_14209_b200 import workloads as W
+import gpu_harness as H
+
+IMPLS = [pytest.param(0, id="default"), pytest.param(mb.FLAG_SIMT_KERNELS, id="simt")]
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2602_14209_b200 import build
+    build.build()
+    assert torch.cuda.is_available()
+    mb.load()
+
+
+@pytest.mark.parametrize("flags", IMPLS)
+def test_cfg1_small_all_elements(oracle_mod, flags):
+    w = W.CONFIGS["cfg1_small"]
+    batch = W.make_batch(w, device="cuda")
+    res = H.run_gpu_block(batch, w, flags=flags)
+    d = H.check_problem(oracle_mod, batch, res, w, 0)
+    print("cfg1", d)
+    assert res["launches"] > 0
+
+
+SMALL = [
+    # (H_q, H_kv, B, N, k, T)  -- ragged tails, N < k, N < one tile, every G and B the sweep uses
+    (8, 2, 32, 1000, 256, 2), (7, 1, 32, 777, 64, 2), (28, 4, 4, 1500, 128, 2), (28, 4, 16, 2049, 300, 2),
+    (14, 2, 64, 1300, 2048, 2), (4, 4, 1, 130, 16, 2), (8, 2, 32, 100, 256, 2), (8, 2, 32, 0, 32, 2),
+    (32, 8, 32, 4097, 512, 3), (8, 1, 64, 3000, 1024, 2),
+]
+
+
+@pytest.mark.parametrize("flags", IMPLS)
+@pytest.mark.parametrize("shape", SMALL, ids=lambda s: "x".join(map(str, s)))
+def test_small_and_ragged_shapes(oracle_mod, flags, shape):
+    H_q, H_kv, B, N, k, T = shape
+    w = W.Workload("small", H_q=H_q, H_kv=H_kv, N=N, B=B, k=k, T=T, n_heavy=min(32, N), seed=3)
+    batch = W.make_batch(w, device="cuda")
+    res = H.run_gpu_block(batch, w, flags=flags)
+    H.check_problem(oracle_mod, batch, res, w, 0)
+
+
+@pytest.mark.parametrize("flags", IMPLS)
+def test_batched_ragged_contiguous_and_paged_agree_with_oracle(oracle_mod, flags):
+    w = W.Workload("ragged", H_q=8, H_kv=2, N=3000, B=32, k=200, T=2, P=5, n_heavy=32, ragged_min=40, page_size=64, seed=5)
+    batch = W.make_batch(w, device="cuda")
+    batch["seq_lens"][1] = 0                                         # one empty prefix in the batch
+    for paged in (False, True):
+        res = H.run_gpu_block(batch, w, flags=flags, paged=paged)
+        for p in range(w.P):
+            H.check_problem(oracle_mod, batch, res, w, p)
+
+
+@pytest.mark.parametrize("flags", IMPLS)
+def test_strided_cache_view(oracle_mod, flags):
+    """The contiguous layout takes arbitrary (8-element aligned) strides: a [P, N, H_kv, d] buffer viewed as [P, H_kv, N, d]."""
+    w = W.Workload("strided", H_q=8, H_kv=2, N=900, B=16, k=100, T=2, P=2, n_heavy=16, seed=9)
+    batch = W.make_batch(w, device="cuda")
+    kc_t = batch["kc"].permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    vc_t = batch["vc"].permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    assert not kc_t.is_contiguous()
+    b2 = dict(batch, kc=kc_t, vc=vc_t)
+    res = H.run_gpu_block(b2, w, flags=flags)
+    for p in range(w.P):
+        H.check_problem(oracle_mod, batch, res, w, p)
+
+
+@pytest.mark.parametrize("flags", IMPLS)
+def test_runs_are_bitwise_reproducible(flags):
+    w = dataclasses.replace(W.CONFIGS["cfg1_small"], N=5000, T=2)
+    batch = W.make_batch(w, device="cuda")
+    a = H.run_gpu_block(batch, w, flags=flags)
+    b = H.run_gpu_block(batch, w, flags=flags)
+    for x, y in zip(a["outs"], b["outs"]):
+        assert np.array_equal(x, y)
+    assert np.array_equal(a["scores"], b["scores"]) and np.array_equal(a["indices"], b["indices"])
+
+
+def test_topk_edge_cases_against_full_sort():
+    """mage_topk alone on crafted score rows: ties, zeros, k = N, k > N, N = 1, ragged lengths."""
+    torch.manual_seed(0)
+    P, H_kv, N_max, k = 3, 2, 5000, 37
+    sc = torch.rand(P, H_kv, N_max, device="cuda")
+    sc[0, 0, ::3] = 0.25                       # many exact ties around the threshold region
+    sc[0, 1] = 0.0                             # all equal: the first k positions win
+    sc[1, 0, :100] = torch.linspace(1, 2, 100, device="cuda")
+    sc[2, 1, 4000:] = 1e-30                    # tiny values
+    lens = torch.tensor([5000, 20, 4999], dtype=torch.int32, device="cuda")
+    idx = torch.empty(P, H_kv, k, dtype=torch.int32, device="cuda")
+    keff = torch.empty(P, dtype=torch.int32, device="cuda")
+    mb.mage_topk(sc, lens, P, H_kv, N_max, k, idx, keff)
+    torch.cuda.synchronize()
+    from helpers import brute_force_topk
+    for p in range(P):
+        n = int(lens[p])
+        assert int(keff[p]) == min(k, n)
+        for h in range(H_kv):
+            ref = brute_force_topk(sc[p, h, :n].double().cpu().numpy(), k)
+            got = idx[p, h].cpu().numpy()
+            assert np.array_equal(got[: len(ref)], ref), (p, h)
+            assert (got[len(ref):] == -1).all()
+
+
+def test_bad_indices_and_pages_are_flagged_not_dereferenced():
+    """Host-made faults: an out-of-range index / page id sets a status bit and the row is skipped; nothing traps."""
+    w = W.Workload("bad", H_q=8, H_kv=2, N=640, B=32, k=64, T=2, n_heavy=16, page_size=64, seed=2)
+    batch = W.make_batch(w, device="cuda")
+    for paged in (False, True):
+        res = H.run_gpu_block(batch, w, paged=paged)
+        ba = res["ba"]
+        good = ba.sparse_step(batch["q"][1], batch["kb"][1], batch["vb"][1]).clone()
+        ba.indices[0, 0, 5] = 1 << 28
+        ba.indices[0, 1, 0] = -7
+        ba.status.zero_()
+        out = ba.sparse_step(batch["q"][1], batch["kb"][1], batch["vb"][1])
+        torch.cuda.synchronize()
+        assert int(ba.status.item()) & mb.DEV_BAD_INDEX
+        assert torch.isfinite(out.float()).all()
+        assert (out.float() - good.float()).abs().max() < 0.1         # one of 64+32 keys dropped per head
+    res = H.run_gpu_block(batch, w, paged=True)
+    res["table"][0, 3] = 10 ** 6
+    ba = res["ba"]
+    ba.status.zero_()
+    ba.exact_select(batch["q"][0], batch["kb"][0], batch["vb"][0])
+    torch.cuda.synchronize()
+    assert int(ba.status.item()) & mb.DEV_BAD_PAGE
+    assert torch.isfinite(ba.out.float()).all()
