@@ -1,0 +1,357 @@
+#!/usr/bin/env python
+"""Benchmark of the MAGE per-block attention path: one "step" = one block of Algorithm 1
+(Step-1 exact attention + block score, top-k on the select stream, T-1 sparse reuse steps)
+over the 28-layer, 128K-context Qwen2.5-7B-shaped workload.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl mage|reference] [--workload NAME] [--simt]
+
+Prints one JSON line (rank 0).  With --impl reference the CPU oracle is timed on the host
+cores on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "per_block_attention_latency"
+UNIT = "ms/block"
+SM_COUNT, FP32_LANES_PER_SM = 148, 128
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"], "bf16_tflops_sustained": p["bf16_tflops_sustained"],
+                "sm_max_mhz": p.get("sm_max_mhz", 1965.0), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0, "source": "fallback"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.rows, self._stop_evt, self.proc = index, [], threading.Event(), None
+
+    def run(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            for line in self.proc.stdout:
+                if self._stop_evt.is_set():
+                    break
+                self.rows.append([x.strip() for x in line.split(",")])
+        except Exception:
+            pass
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.proc is not None:
+            self.proc.terminate()
+        rows = [r for r in self.rows if len(r) >= 7 and r[0].replace(".", "").isdigit()]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        sm = sorted(float(r[0]) for r in rows)
+        reasons = []
+        for i, name in ((3, "hw_slowdown"), (4, "hw_thermal_slowdown"), (5, "sw_thermal_slowdown"), (6, "sw_power_cap")):
+            if any(r[i].lower().startswith("active") for r in rows):
+                reasons.append(name)
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(rows[0][1]), "reasons": reasons, "samples": len(rows),
+                "power_w_max": max(float(r[2]) for r in rows)}
+
+
+def stage_bytes_flops(w, lens):
+    """Algorithmic traffic and work of each stage for one block (all problems).
+
+    Stage 1 must read every cached K and V row once (512 B per cached token per KV head), Q and the block's K/V,
+    and write O and one fp32 score per cached token per KV head.  Its work is a dense (G*B) x N x d contraction
+    done for the attention (QK^T and PV: 4*M*d flops per cached token per KV head) and once more for the score's
+    QK^T (2*M*d).  Stage 3 gathers k rows of K and V per KV head and reads/writes Q, O, the block's K/V and indices.
+    """
+    d, M = w.d, w.M
+    tok = sum(lens)
+    qo = len(lens) * w.H_q * w.B * d * 2
+    kvb = len(lens) * w.H_kv * w.B * d * 2 * 2
+    s1_bytes = tok * w.H_kv * (2 * d * 2 + 4) + 2 * qo + kvb
+    s1_attn_bytes = tok * w.H_kv * 2 * d * 2 + qo + kvb            # the attention kernel alone
+    s1_flops_attn = sum(4 * M * (n + w.B) * d * w.H_kv for n in lens)
+    s1_flops_score = sum(2 * M * n * d * w.H_kv for n in lens)
+    keff = [min(w.k, n) for n in lens]
+    s3_bytes = sum(ke * w.H_kv * (2 * d * 2 + 4) for ke in keff) + 2 * qo + kvb
+    s3_flops = sum(4 * M * (ke + w.B) * d * w.H_kv for ke in keff)
+    return {"s1_bytes": s1_bytes, "s1_attn_bytes": s1_attn_bytes, "s1_flops_attn": s1_flops_attn,
+            "s1_flops_score": s1_flops_score, "s3_bytes": s3_bytes, "s3_flops": s3_flops}
+
+
+def run_reference(args, w):
+    """The CPU oracle, as it stands, on a bounded sample: one KV head of one layer per step, scaled to the whole block."""
+    import numpy as np
+    import oracle
+    from paper_2602_14209_b200 import workloads as W
+    oracle.build()
+    lens = W.seq_lens_for(w)
+    p = max(range(w.P), key=lambda i: lens[i]) if w.ragged_min else 0
+    pr = W.make_problem(w, p, N=lens[p], device="cpu")
+    f = lambda t: t.float().numpy()
+    q = [f(pr["q"][t]) for t in range(w.T)]
+    kb = [f(pr["kb"][t]) for t in range(w.T)]
+    vb = [f(pr["vb"][t]) for t in range(w.T)]
+    Kc, Vc = f(pr["kc"]), f(pr["vc"])
+    head_tokens = lens[p]
+    all_head_tokens = sum(lens)
+    times = []
+    for it in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        oracle.run_block(q, Kc, Vc, kb, vb, w.k)
+        dt = time.perf_counter() - t0
+        if it >= args.warmup:
+            times.append(dt)
+    per_sample = sum(times) / len(times)
+    # the exact pass dominates and is linear in cached tokens x KV heads: scale the sample to the whole block
+    ms_block = per_sample * 1e3 * all_head_tokens / head_tokens
+    cores = oracle.num_threads()
+    sample = (f"problem {p} (one layer/sequence, all {w.H_kv} KV heads, N={head_tokens}) of {w.name}: exact + score + top-k + "
+              f"{w.T - 1} sparse steps; scaled to the whole block by cached tokens ({all_head_tokens / head_tokens:.1f}x)")
+    line = {"impl": "reference", "metric": METRIC, "value": ms_block, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_block, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "H_q": w.H_q, "H_kv": w.H_kv, "d": w.d, "N": w.N, "B": w.B, "k": w.k, "T": w.T, "problems": w.P},
+            "cpu_baseline": {"value": ms_block, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                             "sample_seconds": per_sample},
+            "e2e": {"value": ms_block, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="mage", choices=["mage", "reference"])
+    ap.add_argument("--workload", default="cfg3_qwen_128k_x28")
+    ap.add_argument("--simt", action="store_true", help="force the portable CUDA-core kernels")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-stage-breakdown", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    from paper_2602_14209_b200 import workloads as W
+    w = W.CONFIGS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            args.steps, args.warmup = min(args.steps, 3), min(args.warmup, 1)
+            run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2602_14209_b200 import binding as mb
+    from paper_2602_14209_b200.pipeline import BlockAttention
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    mb.load()
+    peaks = load_peaks()
+
+    # weak scaling: every rank runs its own block of the same shape on its own seeded data (independent problems,
+    # no data-path collective); rank r draws seed + r.
+    import dataclasses
+    w_rank = dataclasses.replace(w, seed=w.seed + rank)
+    batch = W.make_batch(w_rank, device=dev)
+    lens = [int(x) for x in batch["seq_lens"].tolist()]
+    flags = mb.FLAG_SIMT_KERNELS if args.simt else 0
+    if w.page_size:
+        k_pool, v_pool, table, _ = W.to_paged(batch["kc"], batch["vc"], lens, w.page_size, seed=w.seed)
+        batch["kc"] = batch["vc"] = None
+        kv = mb.KVCache(k_pool, v_pool, w.H_q, w.B, seq_lens=batch["seq_lens"], block_table=table, N_max=batch["N_max"], flags=flags)
+    else:
+        kv = mb.KVCache(batch["kc"], batch["vc"], w.H_q, w.B, seq_lens=batch["seq_lens"], flags=flags)
+    ba = BlockAttention(kv, w.k)
+    T = w.T
+    q_d = [batch["q"][t] for t in range(T)]
+    kb_d = [batch["kb"][t] for t in range(T)]
+    vb_d = [batch["vb"][t] for t in range(T)]
+    outs = [torch.empty_like(ba.out) for _ in range(T)]
+    sf = stage_bytes_flops(w, lens)
+    main_stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- timed region 1: inputs resident in HBM ---------------------------------------------------------------
+    n_total = args.warmup + args.steps
+    ev_sets = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n_total)]
+    for i in range(args.warmup):
+        ba.run_block(q_d, kb_d, vb_d, outs, events=ev_sets[i])
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = mb.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        ba.run_block(q_d, kb_d, vb_d, outs, events=ev_sets[args.warmup + i])
+    e1.record()
+    barrier()
+    launches = mb.launch_count() - launches0
+    clocks = sampler.stop()
+    ms_total = e0.elapsed_time(e1)
+    attn_ms = [s[0].elapsed_time(s[1]) for s in ev_sets[args.warmup:]]
+    comb_ms = [s[1].elapsed_time(s[2]) for s in ev_sets[args.warmup:]]
+    score_ms = [s[2].elapsed_time(s[3]) for s in ev_sets[args.warmup:]]
+    status = int(ba.status.item())
+
+    # ---- timed region 2: end to end through the public API with host buffers ------------------------------------
+    # Per block the host hands over each step's Q and block K/V (pinned) and reads back each step's output;
+    # the prefix KV cache is resident state of the serving process, as in the paper's exact block-level caching.
+    q_h = [t.cpu().pin_memory() for t in q_d]
+    kb_h = [t.cpu().pin_memory() for t in kb_d]
+    vb_h = [t.cpu().pin_memory() for t in vb_d]
+    out_h = [torch.empty_like(o, device="cpu").pin_memory() for o in outs]
+    q_s, kb_s, vb_s = [torch.empty_like(t) for t in q_d], [torch.empty_like(t) for t in kb_d], [torch.empty_like(t) for t in vb_d]
+    h2d = sum(t.numel() * 2 for t in q_h + kb_h + vb_h)
+    d2h = sum(t.numel() * 2 for t in out_h)
+
+    def e2e_block():
+        for t in range(T):
+            q_s[t].copy_(q_h[t], non_blocking=True); kb_s[t].copy_(kb_h[t], non_blocking=True); vb_s[t].copy_(vb_h[t], non_blocking=True)
+        ba.run_block(q_s, kb_s, vb_s, outs)
+        for t in range(T):
+            out_h[t].copy_(outs[t], non_blocking=True)
+        main_stream.synchronize()
+
+    e2e_steps = args.steps
+    for _ in range(min(args.warmup, 2)):
+        e2e_block()
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record()
+    for _ in range(e2e_steps):
+        e2e_block()
+    f1.record()
+    barrier()
+    e2e_ms_total = f0.elapsed_time(f1)
+
+    # ---- max over ranks ----------------------------------------------------------------------------------------
+    if world > 1:
+        tt = torch.tensor([ms_total, e2e_ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total, e2e_ms_total = float(tt[0]), float(tt[1])
+        lt = torch.tensor([launches], device=dev, dtype=torch.int64)
+        dist.all_reduce(lt)
+        launches = int(lt[0])
+    ms_per_step = ms_total / args.steps
+    value = ms_per_step / world                 # ms per block over the whole job: each of the N ranks finishes one block per step
+    e2e_value = e2e_ms_total / e2e_steps / world
+
+    # ---- per-stage numbers (rank 0, outside the headline region): sparse step cold/warm, top-k alone -------------
+    stages = {}
+    if rank == 0 and not args.no_stage_breakdown:
+        flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+        def timed(fn, cold, reps=10):
+            ts = []
+            for _ in range(reps):
+                if cold:
+                    flush.fill_(1)
+                a.record(); fn(); b.record(); torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            ts.sort()
+            return ts[len(ts) // 2]
+
+        sp = lambda: ba.sparse_step(q_d[1], kb_d[1], vb_d[1], outs[1])
+        tk = lambda: mb.mage_topk(ba.scores, kv.seq_lens, kv.P, kv.H_kv, kv.N_max, w.k, ba.indices, ba.k_eff)
+        sp(); tk(); torch.cuda.synchronize()
+        sp_cold, sp_warm, tk_ms = timed(sp, True), timed(sp, False), timed(tk, False)
+        s1_ms = (sum(attn_ms) + sum(comb_ms) + sum(score_ms)) / len(attn_ms)
+        stages = {
+            "exact_select_ms": s1_ms, "attn_kernel_ms": sum(attn_ms) / len(attn_ms), "combine_kernel_ms": sum(comb_ms) / len(comb_ms),
+            "score_kernel_ms": sum(score_ms) / len(score_ms),
+            "exact_select_gbs": sf["s1_bytes"] / s1_ms / 1e6, "exact_select_frac_of_8tbs": sf["s1_bytes"] / s1_ms / 1e6 / 8000.0,
+            "exact_select_frac_of_measured_hbm": sf["s1_bytes"] / s1_ms / 1e6 / peaks["hbm_gbs"],
+            "exact_select_tflops": (sf["s1_flops_attn"] + sf["s1_flops_score"]) / s1_ms / 1e9,
+            "topk_ms_alone": tk_ms, "sparse_step_ms_cold_l2": sp_cold, "sparse_step_ms_warm_l2": sp_warm,
+            "sparse_step_gbs_cold": sf["s3_bytes"] / sp_cold / 1e6, "sparse_step_frac_of_8tbs_cold": sf["s3_bytes"] / sp_cold / 1e6 / 8000.0,
+            "sparse_step_frac_of_measured_hbm_cold": sf["s3_bytes"] / sp_cold / 1e6 / peaks["hbm_gbs"],
+            "sparse_step_tflops_cold": sf["s3_flops"] / sp_cold / 1e9,
+            "hbm_roofline_ms_block_at_8tbs": (sf["s1_bytes"] + (T - 1) * sf["s3_bytes"]) / 8e9,
+        }
+        del flush
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (the Step-1 attention kernel) -------------------------------------------
+    attn_avg_ms = sum(attn_ms) / len(attn_ms)
+    if args.simt:
+        peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+        roofline = {"bound": "alu", "kernel": "simt::attn_kernel<kExactPartial>", "achieved": sf["s1_flops_attn"] / attn_avg_ms / 1e9,
+                    "peak": peak, "unit": "TFLOP/s", "peak_source": "148 SMs x 128 fp32 lanes x 2 flop x 1965 MHz (derived)",
+                    "traffic": None}
+    else:
+        roofline = {"bound": "tensor", "kernel": "exact-pass attention kernel", "achieved": sf["s1_flops_attn"] / attn_avg_ms / 1e9,
+                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                    "peak_source": f"bf16 cuBLAS sustained, {peaks['source']}", "traffic": None}
+    roofline["frac"] = roofline["achieved"] / roofline["peak"]
+    roofline["hbm_view"] = {"achieved_gbs": sf["s1_attn_bytes"] / attn_avg_ms / 1e6, "peak_gbs": peaks["hbm_gbs"],
+                            "frac_of_measured": sf["s1_attn_bytes"] / attn_avg_ms / 1e6 / peaks["hbm_gbs"],
+                            "frac_of_8tbs": sf["s1_attn_bytes"] / attn_avg_ms / 1e6 / 8000.0}
+    prof = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(prof):
+        try:
+            roofline["traffic"] = json.load(open(prof)).get("simt" if args.simt else "default", {}).get(w.name)
+        except Exception:
+            pass
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        out = subprocess.run([sys.executable, os.path.abspath(__file__), "--impl", "reference", "--steps", "1", "--warmup", "0",
+                              "--workload", args.workload], capture_output=True, text=True)
+        try:
+            cpu_baseline = json.loads(out.stdout.strip().splitlines()[-1])["cpu_baseline"]
+        except Exception:
+            cpu_baseline = {"value": None, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle", "sample": "failed: " + out.stderr[-200:]}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "H_q": w.H_q, "H_kv": w.H_kv, "d": w.d, "N": w.N, "B": w.B, "k": w.k, "T": w.T,
+                   "problems": w.P, "cached_tokens": sum(lens), "kv_bytes": sum(lens) * w.H_kv * 512,
+                   "l2_policy": "inputs_larger_than_l2 (KV cache streamed every step evicts L2)",
+                   "parallelism": f"replicas x{world} (independent blocks, no collective)", "kernels": "simt" if args.simt else "default"},
+        "clocks": clocks, "gpu_launches": launches, "dev_status": status,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "roofline": roofline, "cpu_baseline": cpu_baseline, "stages": stages,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -110,6 +110,20 @@ mage_status mage_exact_select(const mage_kv_t *kv, const void *q, const void *k_
                               uint32_t *dev_status, void *stream);
 
 /*
+ * The same operation as mage_exact_select (Algorithm 1, Phase 1; Eq. 4), with
+ * CUDA events recorded between its kernels so that a caller can time each one
+ * on the stream it runs on.  `events` is a HOST array of 4 cudaEvent_t handles
+ * (created by the caller with timing enabled), recorded on `stream` in this order:
+ *   [0] before the first kernel, [1] after the attention kernel over prefix + block keys,
+ *   [2] after the kernel that merges the per-chunk partial results,
+ *   [3] after the block-score kernel.
+ * events == NULL behaves exactly like mage_exact_select.
+ */
+mage_status mage_exact_select_events(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk,
+                                     float sm_scale, void *out, float *scores, void *workspace,
+                                     size_t workspace_bytes, uint32_t *dev_status, void *stream, void **events);
+
+/*
  * Top-k selection per KV head (Algorithm 1, "S <- Top-k(alpha)"; Eq. 4).
  *
  *   scores   [P][H_kv][N_max] fp32, non-negative, no NaN

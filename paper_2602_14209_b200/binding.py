@@ -38,7 +38,7 @@ class mage_kv_t(ctypes.Structure):
     ]
 
 
-EXPORTS = ("mage_workspace_bytes", "mage_exact_select", "mage_topk", "mage_sparse_block_attn",
+EXPORTS = ("mage_workspace_bytes", "mage_exact_select", "mage_exact_select_events", "mage_topk", "mage_sparse_block_attn",
            "mage_status_string", "mage_launch_count")
 
 
@@ -55,6 +55,8 @@ def load():
     lib.mage_workspace_bytes.argtypes = [ctypes.POINTER(mage_kv_t), i32]
     lib.mage_exact_select.restype = ctypes.c_int
     lib.mage_exact_select.argtypes = [ctypes.POINTER(mage_kv_t), vp, vp, vp, ctypes.c_float, vp, vp, vp, ctypes.c_size_t, vp, vp]
+    lib.mage_exact_select_events.restype = ctypes.c_int
+    lib.mage_exact_select_events.argtypes = lib.mage_exact_select.argtypes + [ctypes.POINTER(ctypes.c_void_p)]
     lib.mage_topk.restype = ctypes.c_int
     lib.mage_topk.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, ctypes.c_size_t, vp]
     lib.mage_sparse_block_attn.restype = ctypes.c_int
@@ -131,11 +133,24 @@ class KVCache:
         return torch.empty(n, dtype=torch.uint8, device=self.device)
 
 
-def mage_exact_select(kv: KVCache, q, k_blk, v_blk, sm_scale: float, out, scores, workspace, dev_status=None, stream=None):
-    """Step 1 of a block: exact attention into ``out`` and block scores into ``scores`` (see mage.h)."""
-    rc = load().mage_exact_select(ctypes.byref(kv.c), _ptr(q), _ptr(k_blk), _ptr(v_blk), float(sm_scale), _ptr(out),
-                                  _ptr(scores), _ptr(workspace), workspace.numel() * workspace.element_size() if workspace is not None else 0,
-                                  _ptr(dev_status), _stream(stream))
+def mage_exact_select(kv: KVCache, q, k_blk, v_blk, sm_scale: float, out, scores, workspace, dev_status=None, stream=None,
+                      events=None):
+    """Step 1 of a block: exact attention into ``out`` and block scores into ``scores`` (see mage.h).
+
+    ``events``: optional list of four recorded-on-demand ``torch.cuda.Event(enable_timing=True)`` objects; when given,
+    the call goes through ``mage_exact_select_events`` and the library records them between its kernels.
+    """
+    ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    args = (ctypes.byref(kv.c), _ptr(q), _ptr(k_blk), _ptr(v_blk), float(sm_scale), _ptr(out), _ptr(scores), _ptr(workspace),
+            ws_bytes, _ptr(dev_status), _stream(stream))
+    if events is None:
+        rc = load().mage_exact_select(*args)
+    else:
+        for e in events:                 # torch creates the CUDA event lazily, at its first record
+            if not e.cuda_event:
+                e.record()
+        handles = (ctypes.c_void_p * 4)(*[ctypes.c_void_p(e.cuda_event) for e in events])
+        rc = load().mage_exact_select_events(*args, handles)
     if rc != MAGE_OK:
         raise MageError(rc, "mage_exact_select")
 

@@ -85,23 +85,28 @@ static mage_status opt_in_smem(K kernel, size_t bytes) {
 
 static mage_status exact_select_simt(const mage_kv_t *kv, const KvView &view, const Plan &plan, const __nv_bfloat16 *q,
                                      const __nv_bfloat16 *k_blk, const __nv_bfloat16 *v_blk, float sm_scale,
-                                     __nv_bfloat16 *out, float *scores, float *ws, unsigned *dev_status, cudaStream_t st) {
+                                     __nv_bfloat16 *out, float *scores, float *ws, unsigned *dev_status, cudaStream_t st,
+                                     cudaEvent_t *ev) {
     using namespace simt;
     const float scale_log2 = sm_scale * kLog2e;
     auto kern = attn_kernel<Mode::kExactPartial>;
     if (opt_in_smem(kern, kSmemBytes) != MAGE_OK || opt_in_smem(score_kernel, kSmemBytes) != MAGE_OK) return MAGE_ERR_CUDA;
     const int row_tiles = (view.M + kRows - 1) / kRows;
     dim3 grid(row_tiles, plan.n_chunks + 1, kv->P * kv->H_kv);
+    if (ev) cudaEventRecord(ev[0], st);
     kern<<<grid, kThreads, kSmemBytes, st>>>(view, plan, q, k_blk, v_blk, nullptr, nullptr, 0, scale_log2, ws, nullptr, dev_status);
     if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    if (ev) cudaEventRecord(ev[1], st);
     const int rows_total = kv->P * kv->H_kv * view.M;
     combine_kernel<<<(rows_total + 3) / 4, 128, 0, st>>>(view, plan, ws, out);
     if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    if (ev) cudaEventRecord(ev[2], st);
     if (kv->N_max > 0) {
         dim3 sgrid((kv->N_max + kKeys - 1) / kKeys, 1, kv->P * kv->H_kv);
         score_kernel<<<sgrid, kThreads, kSmemBytes, st>>>(view, plan, q, scale_log2, ws, scores, dev_status);
         if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
     }
+    if (ev) cudaEventRecord(ev[3], st);
     return MAGE_OK;
 }
 
@@ -128,9 +133,9 @@ size_t mage_workspace_bytes(const mage_kv_t *kv, int32_t k_max) {
     return make_plan(kv).total_bytes;
 }
 
-mage_status mage_exact_select(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk, float sm_scale,
-                              void *out, float *scores, void *workspace, size_t workspace_bytes, uint32_t *dev_status,
-                              void *stream) {
+mage_status mage_exact_select_events(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk,
+                                     float sm_scale, void *out, float *scores, void *workspace, size_t workspace_bytes,
+                                     uint32_t *dev_status, void *stream, void **events) {
     mage_status why = MAGE_OK;
     if (!valid_kv(kv, &why)) return why;
     if (!q || !k_blk || !v_blk || !out || !workspace || (kv->N_max > 0 && !scores)) return MAGE_ERR_INVALID_ARG;
@@ -140,7 +145,15 @@ mage_status mage_exact_select(const mage_kv_t *kv, const void *q, const void *k_
     const KvView view = make_view(kv);
     return exact_select_simt(kv, view, plan, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_blk),
                              static_cast<const __nv_bfloat16 *>(v_blk), sm_scale, static_cast<__nv_bfloat16 *>(out), scores,
-                             static_cast<float *>(workspace), dev_status, static_cast<cudaStream_t>(stream));
+                             static_cast<float *>(workspace), dev_status, static_cast<cudaStream_t>(stream),
+                             reinterpret_cast<cudaEvent_t *>(events));
+}
+
+mage_status mage_exact_select(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk, float sm_scale,
+                              void *out, float *scores, void *workspace, size_t workspace_bytes, uint32_t *dev_status,
+                              void *stream) {
+    return mage_exact_select_events(kv, q, k_blk, v_blk, sm_scale, out, scores, workspace, workspace_bytes, dev_status,
+                                    stream, nullptr);
 }
 
 mage_status mage_topk(const float *scores, const int32_t *seq_lens, int32_t P, int32_t H_kv, int32_t N_max, int32_t k,

@@ -31,10 +31,11 @@ class BlockAttention:
         self._scores_ready = torch.cuda.Event()
         self._indices_ready = torch.cuda.Event()
 
-    def exact_select(self, q, k_blk, v_blk, out=None, stream=None):
+    def exact_select(self, q, k_blk, v_blk, out=None, stream=None, events=None):
         """Step 1 on ``stream`` (default: current): exact attention -> out, block scores -> self.scores."""
         out = self.out if out is None else out
-        mb.mage_exact_select(self.kv, q, k_blk, v_blk, self.sm_scale, out, self.scores, self.workspace, self.status, stream)
+        mb.mage_exact_select(self.kv, q, k_blk, v_blk, self.sm_scale, out, self.scores, self.workspace, self.status, stream,
+                             events)
         return out
 
     def select_async(self, main_stream=None):
@@ -58,14 +59,14 @@ class BlockAttention:
                                   self.workspace, self.status, stream)
         return out
 
-    def run_block(self, q_steps: Sequence[torch.Tensor], kb_steps, vb_steps, outs: Optional[Sequence[torch.Tensor]] = None):
+    def run_block(self, q_steps: Sequence[torch.Tensor], kb_steps, vb_steps, outs: Optional[Sequence[torch.Tensor]] = None,
+                  events=None):
         """One block: Step 1, asynchronous selection, join, then len(q_steps)-1 reuse steps.  Returns the outputs."""
         T = len(q_steps)
         res = []
-        o = self.exact_select(q_steps[0], kb_steps[0], vb_steps[0], None if outs is None else outs[0])
+        o = self.exact_select(q_steps[0], kb_steps[0], vb_steps[0], None if outs is None else outs[0], events=events)
         res.append(o)
-        if T > 1 or True:
-            self.select_async()
+        self.select_async()
         if T > 1:
             self.join()
         for t in range(1, T):
