@@ -1,9 +1,11 @@
 // Host side of libmage: argument validation, workspace planning and kernel launches behind the C ABI.
+#include <algorithm>
 #include <atomic>
 #include <cstdio>
 
 #include "common.cuh"
 #include "simt_kernels.cuh"
+#include "tc_host.cuh"
 #include "topk.cuh"
 
 namespace mage {
@@ -90,7 +92,7 @@ static mage_status exact_select_simt(const mage_kv_t *kv, const KvView &view, co
     using namespace simt;
     const float scale_log2 = sm_scale * kLog2e;
     auto kern = attn_kernel<Mode::kExactPartial>;
-    if (opt_in_smem(kern, kSmemBytes) != MAGE_OK || opt_in_smem(score_kernel, kSmemBytes) != MAGE_OK) return MAGE_ERR_CUDA;
+    if (opt_in_smem(kern, kSmemBytes) != MAGE_OK || opt_in_smem(simt::score_kernel, kSmemBytes) != MAGE_OK) return MAGE_ERR_CUDA;
     const int row_tiles = (view.M + kRows - 1) / kRows;
     dim3 grid(row_tiles, plan.n_chunks + 1, kv->P * kv->H_kv);
     if (ev) cudaEventRecord(ev[0], st);
@@ -101,9 +103,25 @@ static mage_status exact_select_simt(const mage_kv_t *kv, const KvView &view, co
     combine_kernel<<<(rows_total + 3) / 4, 128, 0, st>>>(view, plan, ws, out);
     if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
     if (ev) cudaEventRecord(ev[2], st);
-    if (kv->N_max > 0) {
+    bool tc_score_done = false;
+    if (tc::eligible(kv)) {
+        CUtensorMap map_q, map_k;
+        if (tc::make_rows_map(&map_q, q, (long long)kv->P * kv->H_q * kv->B) && tc::make_cache_map(&map_k, kv, kv->k_cache) &&
+            opt_in_smem(tc::score_kernel, tc::kScoreSmemBytes) == MAGE_OK) {
+            const int tpc = tc::tiles_per_cta_for((long long)kv->P * kv->H_kv, kv->N_max);
+            const int tiles_head = (kv->N_max + tc::kTile - 1) / tc::kTile;
+            dim3 sgrid((tiles_head + tpc - 1) / tpc, kv->P * kv->H_kv, 1);
+            for (int r0 = 0; r0 < view.M; r0 += 256) {
+                tc::score_kernel<<<sgrid, tc::kScoreThreads, tc::kScoreSmemBytes, st>>>(map_q, map_k, view, plan, r0, std::min(256, view.M - r0),
+                                                                                       tpc, scale_log2, ws, scores, r0 > 0, dev_status);
+                if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+            }
+            tc_score_done = true;
+        }
+    }
+    if (!tc_score_done && kv->N_max > 0) {
         dim3 sgrid((kv->N_max + kKeys - 1) / kKeys, 1, kv->P * kv->H_kv);
-        score_kernel<<<sgrid, kThreads, kSmemBytes, st>>>(view, plan, q, scale_log2, ws, scores, dev_status);
+        simt::score_kernel<<<sgrid, kThreads, kSmemBytes, st>>>(view, plan, q, scale_log2, ws, scores, dev_status);
         if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
     }
     if (ev) cudaEventRecord(ev[3], st);

@@ -1,0 +1,77 @@
+// Host side of the tensor-core path: TMA tensor maps (built per call, passed by value as kernel parameters)
+// and launch geometry.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "tc_kernels.cuh"
+
+namespace mage {
+namespace tc {
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                   const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver entry point is looked up through the runtime, so the library does not link against libcuda.
+inline EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// bf16 tensor of `rank` dims (dim 0 = the 128-element head dimension), boxes of 64 x 64 (x 1 x 1), 128-byte swizzle.
+inline bool make_map(CUtensorMap *m, const void *base, int rank, const cuuint64_t *dims, const cuuint64_t *strides_bytes) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint32_t box[4] = {64, 64, 1, 1}, estr[4] = {1, 1, 1, 1};
+    if (dims[1] < 1) return false;
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), dims, strides_bytes, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// [rows][128] row-major matrix (queries, or the block's own keys / values).
+inline bool make_rows_map(CUtensorMap *m, const void *base, long long rows) {
+    cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)rows}, str[1] = {(cuuint64_t)kD * 2};
+    return make_map(m, base, 2, dims, str);
+}
+
+// The prefix cache as a rank-4 tensor: (d, N_max, H_kv, P) with the caller's strides, or (d, page_size, H_kv, num_pages).
+inline bool make_cache_map(CUtensorMap *m, const mage_kv_t *kv, const void *base) {
+    if (kv->page_size == 0) {
+        cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)kv->N_max, (cuuint64_t)kv->H_kv, (cuuint64_t)kv->P};
+        cuuint64_t str[3] = {(cuuint64_t)kv->stride_n * 2, (cuuint64_t)kv->stride_h * 2, (cuuint64_t)kv->stride_p * 2};
+        return make_map(m, base, 4, dims, str);
+    }
+    cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)kv->page_size, (cuuint64_t)kv->H_kv, (cuuint64_t)kv->num_pages};
+    cuuint64_t str[3] = {(cuuint64_t)kD * 2, (cuuint64_t)kv->page_size * kD * 2, (cuuint64_t)kv->H_kv * kv->page_size * kD * 2};
+    return make_map(m, base, 4, dims, str);
+}
+
+// Whether the tensor-core kernels cover this cache description.
+inline bool eligible(const mage_kv_t *kv) {
+    if (kv->flags & MAGE_FLAG_SIMT_KERNELS) return false;
+    if (kv->N_max < 1) return false;
+    if (kv->page_size != 0 && kv->page_size % 64 != 0) return false;
+    if ((reinterpret_cast<uintptr_t>(kv->k_cache) | reinterpret_cast<uintptr_t>(kv->v_cache)) & 15) return false;
+    return encode_fn() != nullptr;
+}
+
+// Tiles per CTA so that the grid is a whole number of waves over 148 SMs with at most ~48 tiles per CTA.
+inline int tiles_per_cta_for(long long heads, int N_max) {
+    const long long tiles_head = (N_max + kTile - 1) / kTile, total = heads * tiles_head;
+    const long long waves = (total + 148LL * 48 - 1) / (148LL * 48);
+    long long tpc = (total + 148 * waves - 1) / (148 * waves);
+    if (tpc < 1) tpc = 1;
+    if (tpc > tiles_head) tpc = tiles_head;
+    return (int)tpc;
+}
+
+}  // namespace tc
+}  // namespace mage
