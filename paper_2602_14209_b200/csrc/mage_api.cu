@@ -53,7 +53,7 @@ static Plan make_plan(const mage_kv_t *kv) {
     pl.M = kv->H_q / kv->H_kv * kv->B;
     pl.Mw = (int)align_up(pl.M, 128);
     const int64_t heads = (int64_t)kv->P * kv->H_kv;
-    int64_t want = (592 + heads - 1) / heads;
+    int64_t want = (1776 + heads - 1) / heads;
     const int64_t max_chunks = kv->N_max > 0 ? (kv->N_max + 1023) / 1024 : 1;
     if (want > max_chunks) want = max_chunks;
     if (want < 1) want = 1;
@@ -96,8 +96,23 @@ static mage_status exact_select_simt(const mage_kv_t *kv, const KvView &view, co
     const int row_tiles = (view.M + kRows - 1) / kRows;
     dim3 grid(row_tiles, plan.n_chunks + 1, kv->P * kv->H_kv);
     if (ev) cudaEventRecord(ev[0], st);
-    kern<<<grid, kThreads, kSmemBytes, st>>>(view, plan, q, k_blk, v_blk, nullptr, nullptr, 0, scale_log2, ws, nullptr, dev_status);
-    if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    bool tc_attn_done = false;
+    if (tc::eligible(kv)) {
+        tc::AttnMaps maps;
+        auto kern_tc = tc::attn_kernel<false>;
+        if (tc::make_rows_map(&maps.q, q, (long long)kv->P * kv->H_q * kv->B) && tc::make_cache_map(&maps.k, kv, kv->k_cache) &&
+            tc::make_cache_map(&maps.v, kv, kv->v_cache) && tc::make_rows_map(&maps.kb, k_blk, (long long)kv->P * kv->H_kv * kv->B) &&
+            tc::make_rows_map(&maps.vb, v_blk, (long long)kv->P * kv->H_kv * kv->B) && opt_in_smem(kern_tc, tc::kAttnSmemBytes) == MAGE_OK) {
+            dim3 tgrid(plan.n_chunks + 1, (view.M + 255) / 256, kv->P * kv->H_kv);
+            kern_tc<<<tgrid, 320, tc::kAttnSmemBytes, st>>>(maps, view, plan, k_blk, v_blk, nullptr, nullptr, 0, scale_log2, ws, nullptr, dev_status);
+            if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+            tc_attn_done = true;
+        }
+    }
+    if (!tc_attn_done) {
+        kern<<<grid, kThreads, kSmemBytes, st>>>(view, plan, q, k_blk, v_blk, nullptr, nullptr, 0, scale_log2, ws, nullptr, dev_status);
+        if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    }
     if (ev) cudaEventRecord(ev[1], st);
     const int rows_total = kv->P * kv->H_kv * view.M;
     combine_kernel<<<(rows_total + 3) / 4, 128, 0, st>>>(view, plan, ws, out);
@@ -133,6 +148,16 @@ static mage_status sparse_simt(const mage_kv_t *kv, const KvView &view, const Pl
                                const int *k_eff, int k, float sm_scale, __nv_bfloat16 *out, unsigned *dev_status,
                                cudaStream_t st) {
     using namespace simt;
+    if (!(kv->flags & MAGE_FLAG_SIMT_KERNELS) && tc::encode_fn() != nullptr) {
+        tc::AttnMaps maps;
+        auto kern_tc = tc::attn_kernel<true>;
+        if (tc::make_rows_map(&maps.q, q, (long long)kv->P * kv->H_q * kv->B) && opt_in_smem(kern_tc, tc::kAttnSmemBytes) == MAGE_OK) {
+            maps.k = maps.v = maps.kb = maps.vb = maps.q;     // unused by the gather producers
+            dim3 tgrid(1, (view.M + 255) / 256, kv->P * kv->H_kv);
+            kern_tc<<<tgrid, 416, tc::kAttnSmemBytes, st>>>(maps, view, plan, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, nullptr, out, dev_status);
+            return launch_check();
+        }
+    }
     auto kern = attn_kernel<Mode::kSparseFinal>;
     if (opt_in_smem(kern, kSmemBytes) != MAGE_OK) return MAGE_ERR_CUDA;
     dim3 grid((view.M + kRows - 1) / kRows, 1, kv->P * kv->H_kv);

@@ -173,5 +173,369 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
     if (warp == 9) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
 }
 
+
+// ------------------------------------------------------------------------------------------------------------
+// Attention kernel (Algorithm 1: "Attn(Q, K, V, C)" over one chunk of the prefix, and "SparseAttn" over the
+// selected rows): flash-style online softmax with both contractions on tcgen05.
+//
+// One CTA owns up to 256 query rows of one KV head (two 128-row M-tiles, one per softmax warpgroup) and walks
+// 128-key tiles.  Per tile and M-tile:  S = Q K^T  (SS MMA into TMEM, 128 fp32 columns)  ->  the warpgroup
+// reads its rows of S, keeps a running reference maximum and sum per row, writes P = exp2(.) as bf16 over the
+// first 64 columns of S  ->  O += P V  (A operand = P from TMEM, B operand = the V tile in its natural
+// [key][d] layout, i.e. MN-major).  While one warpgroup is in its softmax the tensor pipe works for the other.
+// O stays in TMEM for the whole chunk.  A row rescales its O only when its maximum grew by more than 2^8;
+// that happens between "S(i) complete" and "P(i) ready", when no MMA touches O of that M-tile: tcgen05.commit
+// tracks every MMA issued before it, and PV(i-1) is issued before QK(i).
+//
+// DENSE  (SPARSE = false): K/V tiles arrive by TMA from the cache (or from the block's own keys for the last
+//         chunk index); the result is the unnormalised partial (O, m, l) of the chunk, merged by combine_kernel.
+// SPARSE (SPARSE = true): four producer warps gather the k_eff selected cache rows (then the block's keys) with
+//         16-byte cp.async into the same swizzled layout; the result is the final bf16 output.
+// ------------------------------------------------------------------------------------------------------------
+constexpr int kAttnSlots = 5;                          // ring of K/V tile slots: K(0) V(0) K(1) V(1) ...
+constexpr int kAttnQBytes = 2 * kTileBytes;            // two M-tiles of 128 rows
+constexpr size_t kAttnSmemBytes = 1024 + kAttnQBytes + kAttnSlots * kTileBytes + 512;
+constexpr float kRescaleThreshold = 8.f;               // log2 units
+
+struct AttnMaps { CUtensorMap q, k, v, kb, vb; };
+
+template <bool SPARSE>
+__global__ void __launch_bounds__(SPARSE ? 416 : 320, 1)
+attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const __nv_bfloat16 *__restrict__ k_blk,
+            const __nv_bfloat16 *__restrict__ v_blk, const int *__restrict__ indices, const int *__restrict__ k_eff_arr, int k,
+            float scale_log2, float *__restrict__ ws, __nv_bfloat16 *__restrict__ out, unsigned *status) {
+    using namespace ptx;
+    constexpr int kMmaWarp = SPARSE ? 12 : 9;
+    const int chunk = blockIdx.x, rg = blockIdx.y, z = blockIdx.z, p = z / kv.H_kv, h = z % kv.H_kv;
+    const int N = seq_len_of(kv, p);
+    int n_keys, n_cache, j_begin = 0;
+    bool blk_chunk = false;
+    if (!SPARSE) {
+        if (chunk < plan.n_chunks) {
+            j_begin = chunk * plan.chunk_len;
+            if (j_begin >= N) return;
+            n_keys = n_cache = min(plan.chunk_len, N - j_begin);
+        } else {
+            blk_chunk = true;
+            n_keys = kv.B;
+            n_cache = 0;
+        }
+    } else {
+        n_cache = min(max(k_eff_arr[p], 0), k);
+        n_keys = n_cache + kv.B;
+    }
+    const int n_tiles = (n_keys + kTile - 1) / kTile;
+    const int rows_here = min(256, kv.M - rg * 256), n_mt = rows_here > 128 ? 2 : 1;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t *q_s = base, *kv_s = base + kAttnQBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(kv_s + kAttnSlots * kTileBytes);
+    enum { Q_FULL = 0, FULL = 1, EMPTY = FULL + kAttnSlots, S_FULL = EMPTY + kAttnSlots, P_FULL = S_FULL + 2, O_DONE = P_FULL + 2, N_BARS = O_DONE + 1 };
+    uint32_t *tmem_ptr_s = reinterpret_cast<uint32_t *>(bars + N_BARS);
+    volatile int *abort_s = reinterpret_cast<volatile int *>(tmem_ptr_s + 1);
+    auto bar = [&](int i) { return smem_u32(bars + i); };
+    auto slot_of = [](int L) { return L % kAttnSlots; };
+    auto par_of = [](int L) { return (L / kAttnSlots) & 1; };
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        *abort_s = 0;
+        mbar_init(bar(Q_FULL), 1);
+        for (int s = 0; s < kAttnSlots; ++s) { mbar_init(bar(FULL + s), SPARSE ? 128 : 1); mbar_init(bar(EMPTY + s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(bar(S_FULL + b), 1); mbar_init(bar(P_FULL + b), 128); }
+        mbar_init(bar(O_DONE), 1);
+        fence_mbar_init();
+    }
+    if (warp == kMmaWarp) { tmem_alloc(smem_u32(tmem_ptr_s), 512); tmem_relinquish(); }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_ptr_s;
+
+    if (warp >= 8 && warp != kMmaWarp) {
+        // ------------------------------------------------------------------ producers
+        if (!SPARSE) {
+            if (lane == 0) {
+                prefetch_tensormap(blk_chunk ? &maps.kb : &maps.k);
+                prefetch_tensormap(blk_chunk ? &maps.vb : &maps.v);
+                const int blk_rows_total = kv.P * kv.H_kv * kv.B;
+                int issued = 0;
+                for (int L = 0; L < 2 * n_tiles; ++L) {
+                    const int i = L >> 1, is_v = L & 1, slot = slot_of(L);
+                    if (!mbar_wait(bar(EMPTY + slot), par_of(L) ^ 1, abort_s, status)) break;
+                    mbar_arrive_expect_tx(bar(FULL + slot), kTileBytes);
+                    const uint32_t dst = smem_u32(kv_s + slot * kTileBytes);
+                    for (int kh = 0; kh < 2; ++kh) {
+                        if (!blk_chunk) {
+                            int c1, c2, c3;
+                            cache_box_coords(kv, p, h, j_begin + i * kTile + kh * 64, N, c1, c2, c3, is_v ? nullptr : status);
+                            for (int dh = 0; dh < 2; ++dh)
+                                tma_load_4d(dst + dh * kHalfBytes + kh * kBoxBytes, is_v ? &maps.v : &maps.k, bar(FULL + slot), dh * 64, c1, c2, c3);
+                        } else {
+                            const int row = (i == 0 && kh == 0) ? z * kv.B : blk_rows_total + 64;   // beyond the tensor: zero fill
+                            for (int dh = 0; dh < 2; ++dh)
+                                tma_load_2d(dst + dh * kHalfBytes + kh * kBoxBytes, is_v ? &maps.vb : &maps.kb, bar(FULL + slot), dh * 64, row);
+                        }
+                    }
+                    issued = L + 1;
+                }
+                if (*abort_s) {
+                    for (int L = max(0, issued - kAttnSlots); L < issued; ++L) {
+                        const long long t0 = clock64();
+                        while (!mbar_try_wait(bar(FULL + slot_of(L)), par_of(L)) && clock64() - t0 < 2000000) {}
+                    }
+                }
+            }
+        } else {
+            const int pt = tid - 256, cchunk = pt & 15, r0 = pt >> 4;
+            int prev_slot = -1;
+            bool ok = true;
+            for (int L = 0; L < 2 * n_tiles && ok; ++L) {
+                const int i = L >> 1, is_v = L & 1, slot = slot_of(L);
+                if (!mbar_wait(bar(EMPTY + slot), par_of(L) ^ 1, abort_s, status)) { ok = false; break; }
+                const __nv_bfloat16 *cache = is_v ? kv.v : kv.k, *blk = is_v ? v_blk : k_blk;
+                uint8_t *tile = kv_s + slot * kTileBytes + (cchunk >> 3) * kHalfBytes;
+#pragma unroll 4
+                for (int it = 0; it < 16; ++it) {
+                    const int r = r0 + 8 * it, t = i * kTile + r;
+                    uint8_t *dst = tile + r * 128 + (((cchunk & 7) ^ (r & 7)) << 4);
+                    const __nv_bfloat16 *src = nullptr;
+                    if (t < n_cache) {
+                        const int j = indices[(long long)z * k + t];
+                        if (j >= 0 && j < N) {
+                            const long long off = cache_row_offset(kv, p, h, j, status);
+                            if (off >= 0) src = cache + off + cchunk * 8;
+                        } else if (status) {
+                            atomicOr(status, MAGE_DEV_BAD_INDEX);
+                        }
+                    } else if (t < n_keys) {
+                        src = blk + ((long long)z * kv.B + (t - n_cache)) * kD + cchunk * 8;
+                    }
+                    if (src) cp_async_16(smem_u32(dst), src);
+                    else *reinterpret_cast<uint4 *>(dst) = make_uint4(0, 0, 0, 0);
+                }
+                cp_async_commit();
+                if (prev_slot >= 0) {
+                    cp_async_wait<1>();
+                    fence_proxy_async();
+                    mbar_arrive(bar(FULL + prev_slot));
+                }
+                prev_slot = slot;
+            }
+            cp_async_wait<0>();
+            if (ok && prev_slot >= 0) {
+                fence_proxy_async();
+                mbar_arrive(bar(FULL + prev_slot));
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        // ------------------------------------------------------------------ MMA issue (one lane)
+        if (lane == 0) {
+            prefetch_tensormap(&maps.q);
+            const int q_row0 = (p * kv.H_q + h * kv.G) * kv.B + rg * 256;
+            mbar_arrive_expect_tx(bar(Q_FULL), n_mt * kTileBytes);
+            for (int mt = 0; mt < n_mt; ++mt)
+                for (int dh = 0; dh < 2; ++dh)
+                    for (int rb = 0; rb < 2; ++rb)
+                        tma_load_2d(smem_u32(q_s + mt * kTileBytes + dh * kHalfBytes + rb * kBoxBytes), &maps.q, bar(Q_FULL), dh * 64,
+                                    q_row0 + mt * kTile + rb * 64);
+            const uint32_t idesc_qk = idesc_bf16_f32(kTile, false, false);   // S[128 rows][128 keys]
+            const uint32_t idesc_pv = idesc_bf16_f32(kD, false, true);       // O[128 rows][128 d], V is MN-major
+            const uint32_t q_addr = smem_u32(q_s);
+            auto qk = [&](int i, int mt) {
+                const uint32_t k_addr = smem_u32(kv_s + slot_of(2 * i) * kTileBytes);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t a = smem_desc_sw128(q_addr + mt * kTileBytes + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
+                    const uint64_t b = smem_desc_sw128(k_addr + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
+                    umma_ss(tmem_base + mt * 128, a, b, idesc_qk, ks > 0);
+                }
+            };
+            auto pv = [&](int i, int mt) {
+                const uint32_t v_addr = smem_u32(kv_s + slot_of(2 * i + 1) * kTileBytes);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {      // 16 keys per step: 16 rows of 128 bytes in each d-half
+                    const uint64_t b = smem_desc_sw128(v_addr + ks * 2048, kHalfBytes, 1024);
+                    umma_ts(tmem_base + 256 + mt * 128, tmem_base + mt * 128 + ks * 8, b, idesc_pv, (i > 0 || ks > 0) ? 1u : 0u);
+                }
+            };
+            bool ok = mbar_wait(bar(Q_FULL), 0, abort_s, status);
+            if (ok) ok = mbar_wait(bar(FULL + slot_of(0)), par_of(0), abort_s, status);
+            if (ok) {
+                tc_fence_after_sync();
+                qk(0, 0);
+                umma_commit(bar(S_FULL + 0));
+                if (n_mt == 2) { qk(0, 1); umma_commit(bar(S_FULL + 1)); }
+                umma_commit(bar(EMPTY + slot_of(0)));
+            }
+            for (int i = 0; ok && i < n_tiles; ++i) {
+                const bool more = i + 1 < n_tiles;
+                if (!mbar_wait(bar(FULL + slot_of(2 * i + 1)), par_of(2 * i + 1), abort_s, status)) break;
+                if (!mbar_wait(bar(P_FULL + 0), i & 1, abort_s, status)) break;
+                tc_fence_after_sync();
+                pv(i, 0);
+                if (more) {
+                    if (!mbar_wait(bar(FULL + slot_of(2 * i + 2)), par_of(2 * i + 2), abort_s, status)) break;
+                    tc_fence_after_sync();
+                    qk(i + 1, 0);
+                    umma_commit(bar(S_FULL + 0));
+                }
+                if (n_mt == 2) {
+                    if (!mbar_wait(bar(P_FULL + 1), i & 1, abort_s, status)) break;
+                    tc_fence_after_sync();
+                    pv(i, 1);
+                }
+                umma_commit(bar(EMPTY + slot_of(2 * i + 1)));
+                if (more) {
+                    if (n_mt == 2) { qk(i + 1, 1); umma_commit(bar(S_FULL + 1)); }
+                    umma_commit(bar(EMPTY + slot_of(2 * i + 2)));
+                }
+            }
+            umma_commit(bar(O_DONE));
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax warpgroups
+        const int mt = warp >> 2, w4 = warp & 3;
+        if (mt < n_mt) {
+            const uint32_t lane_off = (uint32_t)(w4 * 32) << 16;
+            const uint32_t tS = tmem_base + mt * 128 + lane_off, tO = tmem_base + 256 + mt * 128 + lane_off;
+            const int row = w4 * 32 + lane, grow = rg * 256 + mt * kTile + row;
+            float m_used = -INFINITY, l = 0.f;
+            bool ok = true;
+            for (int i = 0; i < n_tiles; ++i) {
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(S_FULL + mt), i & 1, abort_s, status))) { ok = false; break; }
+                tc_fence_after_sync();
+                const int valid = min(kTile, n_keys - i * kTile);
+                float mx = -INFINITY;
+#pragma unroll
+                for (int c0 = 0; c0 < kTile; c0 += 32) {
+                    uint32_t r[32];
+                    tmem_ld32(tS + c0, r);
+                    tmem_wait_ld();
+                    if (valid == kTile) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]));
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (c0 + e < valid) mx = fmaxf(mx, __uint_as_float(r[e]));
+                    }
+                }
+                const float mx_s = mx * scale_log2;
+                if (i == 0) {
+                    m_used = mx_s;
+                } else {
+                    const bool need = mx_s > m_used + kRescaleThreshold;
+                    if (__any_sync(0xffffffffu, need)) {
+                        const float m_new = need ? mx_s : m_used;
+                        const float f = ex2(m_used - m_new);
+                        l *= f;
+#pragma unroll
+                        for (int c0 = 0; c0 < kD; c0 += 32) {
+                            uint32_t r[32];
+                            tmem_ld32(tO + c0, r);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * f);
+                            tmem_st32(tO + c0, r);
+                        }
+                        tmem_wait_st();
+                        m_used = m_new;
+                    }
+                }
+                const float neg_m = -m_used;
+                float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+                for (int c0 = 0; c0 < kTile; c0 += 32) {
+                    uint32_t r[32], pk[16];
+                    tmem_ld32(tS + c0, r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        float p0 = ex2(fmaf(__uint_as_float(r[2 * e]), scale_log2, neg_m));
+                        float p1 = ex2(fmaf(__uint_as_float(r[2 * e + 1]), scale_log2, neg_m));
+                        if (valid != kTile) {
+                            if (c0 + 2 * e >= valid) p0 = 0.f;
+                            if (c0 + 2 * e + 1 >= valid) p1 = 0.f;
+                        }
+                        l0 += p0;
+                        l1 += p1;
+                        pk[e] = pack_bf16x2(p0, p1);
+                    }
+                    tmem_st16(tS + (c0 >> 1), pk);
+                }
+                l += l0 + l1;
+                tmem_wait_st();
+                if (!SPARSE && valid != kTile && mt == 0) {
+                    // Last tile of the prefix: cache rows past the end may hold anything (even NaN patterns), and
+                    // 0 * NaN would poison O.  Zero those V rows in shared memory before the PV MMA may start.
+                    const int Lv = 2 * i + 1;
+                    if (!__all_sync(0xffffffffu, mbar_wait(bar(FULL + slot_of(Lv)), par_of(Lv), abort_s, status))) { ok = false; break; }
+                    if (row >= valid) {
+                        uint8_t *vrow = kv_s + slot_of(Lv) * kTileBytes + row * 128;
+#pragma unroll
+                        for (int q4 = 0; q4 < 8; ++q4) {
+                            *reinterpret_cast<uint4 *>(vrow + q4 * 16) = make_uint4(0, 0, 0, 0);
+                            *reinterpret_cast<uint4 *>(vrow + kHalfBytes + q4 * 16) = make_uint4(0, 0, 0, 0);
+                        }
+                    }
+                    fence_proxy_async();
+                }
+                tc_fence_before_sync();
+                mbar_arrive(bar(P_FULL + mt));
+            }
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(O_DONE), 0, abort_s, status));
+            if (ok) {
+                tc_fence_after_sync();
+                const bool row_ok = grow < kv.M;
+                if (!SPARSE) {
+                    const size_t item = (size_t)z * (plan.n_chunks + 1) + chunk;
+                    float *po = ws + plan.off_part_o + (item * plan.Mw + grow) * kD;
+#pragma unroll
+                    for (int c0 = 0; c0 < kD; c0 += 32) {
+                        uint32_t r[32];
+                        tmem_ld32(tO + c0, r);
+                        tmem_wait_ld();
+                        if (row_ok) {
+#pragma unroll
+                            for (int e = 0; e < 32; e += 4)
+                                *reinterpret_cast<uint4 *>(po + c0 + e) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
+                        }
+                    }
+                    if (row_ok) {
+                        float *pml = ws + plan.off_part_ml + (item * plan.Mw + grow) * 2;
+                        pml[0] = m_used;
+                        pml[1] = l;
+                    }
+                } else {
+                    const float inv = 1.f / l;
+                    __nv_bfloat16 *po = out + ((long long)(p * kv.H_q + h * kv.G) * kv.B + grow) * kD;
+#pragma unroll
+                    for (int c0 = 0; c0 < kD; c0 += 32) {
+                        uint32_t r[32];
+                        tmem_ld32(tO + c0, r);
+                        tmem_wait_ld();
+                        if (row_ok) {
+#pragma unroll
+                            for (int e = 0; e < 32; e += 8) {
+                                uint4 v;
+                                v.x = pack_bf16x2(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
+                                v.y = pack_bf16x2(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+                                v.z = pack_bf16x2(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
+                                v.w = pack_bf16x2(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
+                                *reinterpret_cast<uint4 *>(po + c0 + e) = v;
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == kMmaWarp) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
+}
+
 }  // namespace tc
 }  // namespace mage
