@@ -155,6 +155,32 @@ mage_status mage_sparse_block_attn(const mage_kv_t *kv, const void *q, const voi
                                    void *out, void *workspace, size_t workspace_bytes, uint32_t *dev_status,
                                    void *stream);
 
+/*
+ * Step 1 of a block for callers that cannot hand over a workspace (the paper has no counterpart; this is a
+ * packaging variant of mage_exact_select, same arithmetic, same kernels).
+ *
+ * Some hosts of this library may not allocate device memory at the point where they call it: an inference
+ * runtime that carves up all of its memory at start-up and forbids cudaMalloc afterwards, a plugin that runs
+ * inside someone else's memory pool, code on a latency path where an allocation would stall the device.  For
+ * them this entry point takes no workspace argument: the partial results and per-row normalisers that
+ * mage_exact_select keeps in the caller's workspace live in an array that is part of the library image itself
+ * (a file-scope __device__ array of MAGE_STATIC_SCRATCH_BYTES = 32 MiB, held by every GPU that loads the library
+ * until the process exits).  Inputs and outputs are still the caller's.
+ *
+ *   - A description whose mage_workspace_bytes() exceeds MAGE_STATIC_SCRATCH_BYTES is rejected with
+ *     MAGE_ERR_WORKSPACE (and a line on stderr); nothing is launched.  As a guide, one Qwen2.5-7B-shaped layer
+ *     with a 32K-token prefix needs about 18 MB; a 28-layer 128K batch does not fit.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device
+ *     current) and remembers it; make that first call outside any stream capture.
+ *   - The call performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ *   - All calls on a device share the one array, which simply keeps whatever the last call left in it.  Nothing
+ *     in it has to start at zero: the kernels write every element they later read.  Two calls that can overlap
+ *     on the GPU (different streams, no ordering between them) would race on it; order them.
+ */
+#define MAGE_STATIC_SCRATCH_BYTES (32u << 20)
+mage_status mage_exact_select_static(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk,
+                                     float sm_scale, void *out, float *scores, uint32_t *dev_status, void *stream);
+
 /* Static, human-readable name of a status code. */
 const char *mage_status_string(mage_status s);
 

@@ -38,7 +38,7 @@ class mage_kv_t(ctypes.Structure):
     ]
 
 
-EXPORTS = ("mage_workspace_bytes", "mage_exact_select", "mage_exact_select_events", "mage_topk", "mage_sparse_block_attn",
+EXPORTS = ("mage_workspace_bytes", "mage_exact_select", "mage_exact_select_events", "mage_exact_select_static", "mage_topk", "mage_sparse_block_attn",
            "mage_status_string", "mage_launch_count")
 
 
@@ -57,6 +57,8 @@ def load():
     lib.mage_exact_select.argtypes = [ctypes.POINTER(mage_kv_t), vp, vp, vp, ctypes.c_float, vp, vp, vp, ctypes.c_size_t, vp, vp]
     lib.mage_exact_select_events.restype = ctypes.c_int
     lib.mage_exact_select_events.argtypes = lib.mage_exact_select.argtypes + [ctypes.POINTER(ctypes.c_void_p)]
+    lib.mage_exact_select_static.restype = ctypes.c_int
+    lib.mage_exact_select_static.argtypes = [ctypes.POINTER(mage_kv_t), vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
     lib.mage_topk.restype = ctypes.c_int
     lib.mage_topk.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, ctypes.c_size_t, vp]
     lib.mage_sparse_block_attn.restype = ctypes.c_int
@@ -153,6 +155,22 @@ def mage_exact_select(kv: KVCache, q, k_blk, v_blk, sm_scale: float, out, scores
         rc = load().mage_exact_select_events(*args, handles)
     if rc != MAGE_OK:
         raise MageError(rc, "mage_exact_select")
+
+
+STATIC_SCRATCH_BYTES = 32 << 20
+
+
+def mage_exact_select_static(kv: KVCache, q, k_blk, v_blk, sm_scale: float, out, scores, dev_status=None, stream=None):
+    """Step 1 without a caller workspace: the scratch is a fixed array inside the library (see mage.h).
+
+    For hosts that may not allocate device memory when they call.  Descriptions that need more than
+    STATIC_SCRATCH_BYTES are refused with MAGE_ERR_WORKSPACE.  Calls on one device share the scratch, so
+    calls that could overlap on the GPU must be ordered by the caller.
+    """
+    rc = load().mage_exact_select_static(ctypes.byref(kv.c), _ptr(q), _ptr(k_blk), _ptr(v_blk), float(sm_scale), _ptr(out),
+                                         _ptr(scores), _ptr(dev_status), _stream(stream))
+    if rc != MAGE_OK:
+        raise MageError(rc, "mage_exact_select_static")
 
 
 def mage_topk(scores, seq_lens, P: int, H_kv: int, N_max: int, k: int, indices, k_eff, stream=None):

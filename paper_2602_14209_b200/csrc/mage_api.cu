@@ -222,6 +222,36 @@ mage_status mage_sparse_block_attn(const mage_kv_t *kv, const void *q, const voi
                        dev_status, static_cast<cudaStream_t>(stream));
 }
 
+// Scratch for mage_exact_select_static.  In host code this name is only a handle for the runtime, not a device
+// address: the address is looked up once per device below and that pointer is what the kernels receive.
+static __device__ __align__(256) unsigned char g_static_scratch[MAGE_STATIC_SCRATCH_BYTES];
+static void *g_static_scratch_addr[64] = {};
+
+mage_status mage_exact_select_static(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk,
+                                     float sm_scale, void *out, float *scores, uint32_t *dev_status, void *stream) {
+    mage_status why = MAGE_OK;
+    if (!valid_kv(kv, &why)) return why;
+    const size_t need = make_plan(kv).total_bytes;
+    if (need > (size_t)MAGE_STATIC_SCRATCH_BYTES) {
+        std::fprintf(stderr, "libmage: mage_exact_select_static needs %zu bytes of scratch for this description, the built-in "
+                             "array holds %u; use mage_exact_select with a caller workspace\n", need, (unsigned)MAGE_STATIC_SCRATCH_BYTES);
+        return MAGE_ERR_WORKSPACE;
+    }
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MAGE_ERR_CUDA;
+    if (!g_static_scratch_addr[dev]) {      // set-up, once per device, with that device current
+        void *addr = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&addr, g_static_scratch);
+        if (e != cudaSuccess || !addr) {
+            std::fprintf(stderr, "libmage: cudaGetSymbolAddress(static scratch) failed: %s\n", cudaGetErrorString(e));
+            return MAGE_ERR_CUDA;
+        }
+        g_static_scratch_addr[dev] = addr;
+    }
+    return mage_exact_select_events(kv, q, k_blk, v_blk, sm_scale, out, scores, g_static_scratch_addr[dev],
+                                    (size_t)MAGE_STATIC_SCRATCH_BYTES, dev_status, stream, nullptr);
+}
+
 const char *mage_status_string(mage_status s) {
     switch (s) {
         case MAGE_OK: return "MAGE_OK";
