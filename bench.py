@@ -37,39 +37,60 @@ def load_peaks():
 
 
 class ClockSampler(threading.Thread):
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples SM clock and clock-event (throttle) reasons through NVML every few ms while the timed region runs.
 
-    def __init__(self, index: int):
+    Read-only queries; nothing on the GPU is changed.  Falls back to one `nvidia-smi` query if NVML is unavailable.
+    """
+    REASONS = (("hw_slowdown", 0x8), ("hw_thermal_slowdown", 0x40), ("sw_thermal_slowdown", 0x20), ("sw_power_cap", 0x4))
+
+    def __init__(self, index: int, period_s: float = 0.004):
         super().__init__(daemon=True)
-        self.index, self.rows, self._stop_evt, self.proc = index, [], threading.Event(), None
+        self.index, self.period, self.samples, self._stop_evt = index, period_s, [], threading.Event()
+        self.max_mhz, self.nvml = None, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nvml = pynvml
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nvml = None
 
     def run(self):
-        try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
-                                          "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            for line in self.proc.stdout:
-                if self._stop_evt.is_set():
-                    break
-                self.rows.append([x.strip() for x in line.split(",")])
-        except Exception:
-            pass
+        if self.nvml is None:
+            return
+        n = self.nvml
+        while not self._stop_evt.is_set():
+            try:
+                mhz = n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM)
+                try:
+                    mask = n.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+                except Exception:
+                    mask = n.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle)
+                try:
+                    watts = n.nvmlDeviceGetPowerUsage(self.handle) / 1000.0
+                except Exception:
+                    watts = 0.0
+                self.samples.append((float(mhz), int(mask), watts))
+            except Exception:
+                pass
+            time.sleep(self.period)
 
     def stop(self):
         self._stop_evt.set()
-        if self.proc is not None:
-            self.proc.terminate()
-        rows = [r for r in self.rows if len(r) >= 7 and r[0].replace(".", "").isdigit()]
-        if not rows:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        sm = sorted(float(r[0]) for r in rows)
-        reasons = []
-        for i, name in ((3, "hw_slowdown"), (4, "hw_thermal_slowdown"), (5, "sw_thermal_slowdown"), (6, "sw_power_cap")):
-            if any(r[i].lower().startswith("active") for r in rows):
-                reasons.append(name)
-        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(rows[0][1]), "reasons": reasons, "samples": len(rows),
-                "power_w_max": max(float(r[2]) for r in rows)}
+        if self.nvml is not None:
+            self.join(timeout=1.0)
+        if not self.samples:
+            try:
+                out = subprocess.run(["nvidia-smi", "--query-gpu=clocks.sm,clocks.max.sm", "--format=csv,noheader,nounits", "-i",
+                                      str(self.index)], capture_output=True, text=True, timeout=10).stdout.split(",")
+                return {"sm_mhz": float(out[0]), "sm_max_mhz": float(out[1]), "reasons": [], "samples": 1, "source": "nvidia-smi after the run"}
+            except Exception:
+                return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        sm = sorted(x[0] for x in self.samples)
+        reasons = [name for name, bit in self.REASONS if any(x[1] & bit for x in self.samples)]
+        return {"sm_mhz": sm[len(sm) // 2], "sm_min_mhz": sm[0], "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples": len(self.samples), "power_w_max": max(x[2] for x in self.samples), "source": "nvml"}
 
 
 def stage_bytes_flops(w, lens):
@@ -138,8 +159,8 @@ def run_reference(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="mage", choices=["mage", "reference"])
     ap.add_argument("--workload", default="cfg3_qwen_128k_x28")
     ap.add_argument("--simt", action="store_true", help="force the portable CUDA-core kernels")
