@@ -164,6 +164,8 @@ def main():
     ap.add_argument("--impl", default="mage", choices=["mage", "reference"])
     ap.add_argument("--workload", default="cfg3_qwen_128k_x28")
     ap.add_argument("--simt", action="store_true", help="force the portable CUDA-core kernels")
+    ap.add_argument("--P", type=int, default=None, help="override the number of problems (layers/sequences) of the workload")
+    ap.add_argument("--N", type=int, default=None, help="override the prefix length of the workload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-stage-breakdown", action="store_true")
     args = ap.parse_args()
@@ -171,6 +173,9 @@ def main():
 
     from paper_2602_14209_b200 import workloads as W
     w = W.CONFIGS[args.workload]
+    if args.P is not None or args.N is not None:
+        import dataclasses as _dc
+        w = _dc.replace(w, P=args.P or w.P, N=args.N or w.N, name=f"{w.name}[P={args.P or w.P},N={args.N or w.N}]")
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -351,7 +356,8 @@ def main():
     cpu_baseline = None
     if not args.no_cpu_baseline:
         out = subprocess.run([sys.executable, os.path.abspath(__file__), "--impl", "reference", "--steps", "1", "--warmup", "0",
-                              "--workload", args.workload], capture_output=True, text=True)
+                              "--workload", args.workload] + (["--P", str(args.P)] if args.P else []) + (["--N", str(args.N)] if args.N else []),
+                             capture_output=True, text=True)
         try:
             cpu_baseline = json.loads(out.stdout.strip().splitlines()[-1])["cpu_baseline"]
         except Exception:

@@ -102,9 +102,9 @@ static mage_status exact_select_simt(const mage_kv_t *kv, const KvView &view, co
         auto kern_tc = tc::attn_kernel<false>;
         if (tc::make_rows_map(&maps.q, q, (long long)kv->P * kv->H_q * kv->B) && tc::make_cache_map(&maps.k, kv, kv->k_cache) &&
             tc::make_cache_map(&maps.v, kv, kv->v_cache) && tc::make_rows_map(&maps.kb, k_blk, (long long)kv->P * kv->H_kv * kv->B) &&
-            tc::make_rows_map(&maps.vb, v_blk, (long long)kv->P * kv->H_kv * kv->B) && opt_in_smem(kern_tc, tc::kAttnSmemBytes) == MAGE_OK) {
+            tc::make_rows_map(&maps.vb, v_blk, (long long)kv->P * kv->H_kv * kv->B) && opt_in_smem(kern_tc, tc::kAttnSmemBytesDense) == MAGE_OK) {
             dim3 tgrid(plan.n_chunks + 1, (view.M + 255) / 256, kv->P * kv->H_kv);
-            kern_tc<<<tgrid, 320, tc::kAttnSmemBytes, st>>>(maps, view, plan, k_blk, v_blk, nullptr, nullptr, 0, scale_log2, ws, nullptr, dev_status);
+            kern_tc<<<tgrid, 320, tc::kAttnSmemBytesDense, st>>>(maps, view, plan, k_blk, v_blk, nullptr, nullptr, 0, scale_log2, ws, nullptr, dev_status);
             if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
             tc_attn_done = true;
         }
@@ -151,10 +151,10 @@ static mage_status sparse_simt(const mage_kv_t *kv, const KvView &view, const Pl
     if (!(kv->flags & MAGE_FLAG_SIMT_KERNELS) && tc::encode_fn() != nullptr) {
         tc::AttnMaps maps;
         auto kern_tc = tc::attn_kernel<true>;
-        if (tc::make_rows_map(&maps.q, q, (long long)kv->P * kv->H_q * kv->B) && opt_in_smem(kern_tc, tc::kAttnSmemBytes) == MAGE_OK) {
+        if (tc::make_rows_map(&maps.q, q, (long long)kv->P * kv->H_q * kv->B) && opt_in_smem(kern_tc, tc::kAttnSmemBytesSparse) == MAGE_OK) {
             maps.k = maps.v = maps.kb = maps.vb = maps.q;     // unused by the gather producers
             dim3 tgrid(1, (view.M + 255) / 256, kv->P * kv->H_kv);
-            kern_tc<<<tgrid, 416, tc::kAttnSmemBytes, st>>>(maps, view, plan, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, nullptr, out, dev_status);
+            kern_tc<<<tgrid, 416, tc::kAttnSmemBytesSparse, st>>>(maps, view, plan, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, nullptr, out, dev_status);
             return launch_check();
         }
     }

@@ -116,6 +116,18 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
         : "r"(taddr)
         : "memory");
 }
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld(uint32_t (&r)[8]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7])
+                 :
+                 : "memory");
+}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
@@ -136,6 +148,24 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         : "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Same wait, tied to the destination registers of an earlier load so that no use of them can be scheduled above it
+// (needed when the load was issued well before, with other work in between).
+__device__ __forceinline__ void tmem_wait_ld(uint32_t (&r)[32]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                   "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
+                   "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
+                   "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld(uint32_t (&r)[16]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                   "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+                 :
+                 : "memory");
+}
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // ---------------------------------------------------------------- tcgen05.mma (bf16 x bf16 -> fp32, one CTA)
@@ -180,6 +210,78 @@ __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+// ---------------------------------------------------------------- packed fp32 pairs (two lanes per instruction)
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &a, float &b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+// 2^x for NP pairs of values without the special-function unit, so that it can run beside ex2() on other elements:
+// clamp to >= -126, round to the nearest integer n by adding 1.5*2^23, evaluate a degree-5 minimax polynomial of
+// 2^f on f = x - n in [-0.5, 0.5] (relative error 2.4e-7, the same as ex2.approx), add n to the exponent field.
+// Written stage by stage so that the NP dependency chains are interleaved in program order.  On B200 this route
+// costs ~13 issue cycles per element against 8 cycles of MUFU, so it only pays for a minority of the elements.
+template <int NP>
+__device__ __forceinline__ void ex2_poly2_n(uint64_t (&x)[NP]) {
+    const float kMagic = 12582912.f;
+    const uint64_t magic = pack2(kMagic, kMagic), neg_magic = pack2(-kMagic, -kMagic), neg_one = pack2(-1.f, -1.f);
+    uint64_t t[NP], p[NP];
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+        float a, b;
+        unpack2(x[i], a, b);
+        x[i] = pack2(fmaxf(a, -126.f), fmaxf(b, -126.f));
+    }
+#pragma unroll
+    for (int i = 0; i < NP; ++i) t[i] = add2(x[i], magic);
+#pragma unroll
+    for (int i = 0; i < NP; ++i) p[i] = add2(t[i], neg_magic);
+#pragma unroll
+    for (int i = 0; i < NP; ++i) x[i] = fma2(p[i], neg_one, x[i]);          // f = x - n
+    const uint64_t c5 = pack2(0.0013276466634124517f, 0.0013276466634124517f), c4 = pack2(0.009675540961325169f, 0.009675540961325169f),
+                   c3 = pack2(0.05550713464617729f, 0.05550713464617729f), c2 = pack2(0.24022120237350464f, 0.24022120237350464f),
+                   c1 = pack2(0.6931469440460205f, 0.6931469440460205f), c0 = pack2(1.0000001192092896f, 1.0000001192092896f);
+#pragma unroll
+    for (int i = 0; i < NP; ++i) p[i] = fma2(c5, x[i], c4);
+#pragma unroll
+    for (int i = 0; i < NP; ++i) p[i] = fma2(p[i], x[i], c3);
+#pragma unroll
+    for (int i = 0; i < NP; ++i) p[i] = fma2(p[i], x[i], c2);
+#pragma unroll
+    for (int i = 0; i < NP; ++i) p[i] = fma2(p[i], x[i], c1);
+#pragma unroll
+    for (int i = 0; i < NP; ++i) p[i] = fma2(p[i], x[i], c0);
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+        float p0, p1, t0, t1;
+        unpack2(p[i], p0, p1);
+        unpack2(t[i], t0, t1);
+        p0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
+        p1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
+        x[i] = pack2(p0, p1);
+    }
+}
+template <int NP>
+__device__ __forceinline__ void ex2_mufu2_n(uint64_t (&x)[NP]) {
+    float a[NP], b[NP];
+#pragma unroll
+    for (int i = 0; i < NP; ++i) unpack2(x[i], a[i], b[i]);
+#pragma unroll
+    for (int i = 0; i < NP; ++i) { a[i] = ex2(a[i]); b[i] = ex2(b[i]); }
+#pragma unroll
+    for (int i = 0; i < NP; ++i) x[i] = pack2(a[i], b[i]);
 }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;

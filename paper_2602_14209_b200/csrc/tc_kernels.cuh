@@ -39,12 +39,18 @@ __device__ __forceinline__ void cache_box_coords(const KvView &kv, int p, int h,
 // Block-score kernel (Eq. 4): score[j] = 1/M * sum_r exp2(scale_log2 * <q_r, k_j> - lse2_r).
 // Orientation: keys are the MMA M dimension (TMEM lanes), query rows the N dimension (TMEM columns), so each
 // thread owns one key and its sum over rows needs no cross-thread reduction.  One CTA walks `tiles_per_cta`
-// consecutive 128-key tiles of one KV head; S^T tiles are double-buffered in TMEM, one buffer per warpgroup.
+// consecutive 128-key tiles of one KV head; S^T tiles are double-buffered in TMEM.
+// The kernel is bound by the special-function unit (128*M exponentials per tile at 16 per clock per SM, against
+// 4*M clocks of MMA), so the job of the layout is to keep that unit fed: kScoreWgs warpgroups (four warps per
+// scheduler) all work on every tile, each on a slice of the columns (query rows); warpgroups 1.. hand their 128
+// partial sums to warpgroup 0 through shared memory, which adds them in a fixed order.
 // ------------------------------------------------------------------------------------------------------------
 constexpr int kScoreStages = 4;
-constexpr int kScoreThreads = 320;
+constexpr int kScoreWgs = 4;
+constexpr int kScoreThreads = kScoreWgs * 128 + 64;
+constexpr int kScoreProducerWarp = kScoreWgs * 4, kScoreMmaWarp = kScoreWgs * 4 + 1;
 constexpr int kScoreQBytes = 2 * 256 * 128;           // up to 256 query rows, two d-halves
-constexpr size_t kScoreSmemBytes = 1024 + kScoreQBytes + kScoreStages * kTileBytes + 256 * sizeof(float) + 256;
+constexpr size_t kScoreSmemBytes = 1024 + kScoreQBytes + kScoreStages * kTileBytes + (256 + 2 * (kScoreWgs - 1) * 128) * sizeof(float) + 256;
 
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, KvView kv, Plan plan,
@@ -62,9 +68,10 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *q_s = base, *k_s = base + kScoreQBytes;
     float *neg_lse_s = reinterpret_cast<float *>(k_s + kScoreStages * kTileBytes);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(neg_lse_s + 256);
-    // barrier indices
-    enum { Q_FULL = 0, FULL = 1, EMPTY = FULL + kScoreStages, T_FULL = EMPTY + kScoreStages, T_EMPTY = T_FULL + 2, N_BARS = T_EMPTY + 2 };
+    float *part_s = neg_lse_s + 256;                   // [2][kScoreWgs-1][128] partial sums of warpgroups 1..
+    uint64_t *bars = reinterpret_cast<uint64_t *>(part_s + 2 * (kScoreWgs - 1) * 128);
+    enum { Q_FULL = 0, FULL = 1, EMPTY = FULL + kScoreStages, T_FULL = EMPTY + kScoreStages, T_EMPTY = T_FULL + 2,
+           P_FULL = T_EMPTY + 2, P_EMPTY = P_FULL + 2, N_BARS = P_EMPTY + 2 };
     uint32_t *tmem_ptr_s = reinterpret_cast<uint32_t *>(bars + N_BARS);
     volatile int *abort_s = reinterpret_cast<volatile int *>(tmem_ptr_s + 1);
     auto bar = [&](int i) { return smem_u32(bars + i); };
@@ -76,17 +83,22 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
         *abort_s = 0;
         mbar_init(bar(Q_FULL), 1);
         for (int s = 0; s < kScoreStages; ++s) { mbar_init(bar(FULL + s), 1); mbar_init(bar(EMPTY + s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(bar(T_FULL + b), 1); mbar_init(bar(T_EMPTY + b), 128); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar(T_FULL + b), 1);
+            mbar_init(bar(T_EMPTY + b), kScoreWgs * 128);
+            mbar_init(bar(P_FULL + b), (kScoreWgs - 1) * 128);
+            mbar_init(bar(P_EMPTY + b), 128);
+        }
         fence_mbar_init();
     }
-    if (warp == 9) { tmem_alloc(smem_u32(tmem_ptr_s), 512); tmem_relinquish(); }
+    if (warp == kScoreMmaWarp) { tmem_alloc(smem_u32(tmem_ptr_s), 512); tmem_relinquish(); }
     if (tid < 256) neg_lse_s[tid] = tid < rows ? ws[plan.off_neg_lse + (size_t)z * plan.Mw + row_begin + tid] : 0.f;
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_ptr_s;
 
-    if (warp == 8) {
+    if (warp == kScoreProducerWarp) {
         if (lane == 0) {
             prefetch_tensormap(&map_q);
             prefetch_tensormap(&map_k);
@@ -116,7 +128,7 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                 }
             }
         }
-    } else if (warp == 9) {
+    } else if (warp == kScoreMmaWarp) {
         if (lane == 0) {
             const uint32_t idesc = idesc_bf16_f32(n_mma, false, false);
             bool ok = mbar_wait(bar(Q_FULL), 0, abort_s, status);
@@ -137,42 +149,78 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
             }
         }
     } else {
-        const int wg = warp >> 2, w4 = warp & 3;
+        const int wg = warp >> 2, w4 = warp & 3, key = w4 * 32 + lane;
         const float inv_m = 1.f / (float)kv.M;
         float *srow = scores + (size_t)z * kv.N_max;
-        for (int i = wg; i < n_my; i += 2) {
-            const int ub = i >> 1;
-            if (!__all_sync(0xffffffffu, mbar_wait(bar(T_FULL + wg), ub & 1, abort_s, status))) break;
+        // column slice of this warpgroup, in units of 8 columns
+        const int per = (((rows + kScoreWgs - 1) / kScoreWgs) + 7) & ~7;
+        const int col_lo = min(rows, wg * per), col_hi = min(rows, col_lo + per);
+        const uint64_t c2 = pack2(scale_log2, scale_log2);
+        for (int i = 0; i < n_my; ++i) {
+            const int buf = i & 1, ub = i >> 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(T_FULL + buf), ub & 1, abort_s, status))) break;
             tc_fence_after_sync();
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            const uint32_t taddr = tmem_base + wg * 256 + ((uint32_t)(w4 * 32) << 16);
-            for (int c0 = 0; c0 < rows; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld32(taddr + c0, r);
-                tmem_wait_ld();
-                if (c0 + 32 <= rows) {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) acc[e & 3] += ex2(fmaf(__uint_as_float(r[e]), scale_log2, neg_lse_s[c0 + e]));
+            float tail = 0.f;
+            uint64_t acc_a = pack2(0.f, 0.f), acc_b = acc_a;
+            const uint32_t taddr = tmem_base + buf * 256 + ((uint32_t)(w4 * 32) << 16);
+            // one unit = 8 columns = 4 pairs; the TMEM load of the next unit is in flight while this one is processed
+            auto unit = [&](const uint32_t (&r)[8], int c0) {
+                if (c0 + 8 <= col_hi) {
+                    const float4 *nl4 = reinterpret_cast<const float4 *>(neg_lse_s + c0);
+                    const float4 n0 = nl4[0], n1 = nl4[1];
+                    uint64_t x[4];
+                    x[0] = fma2(pack2(__uint_as_float(r[0]), __uint_as_float(r[1])), c2, pack2(n0.x, n0.y));
+                    x[1] = fma2(pack2(__uint_as_float(r[2]), __uint_as_float(r[3])), c2, pack2(n0.z, n0.w));
+                    x[2] = fma2(pack2(__uint_as_float(r[4]), __uint_as_float(r[5])), c2, pack2(n1.x, n1.y));
+                    x[3] = fma2(pack2(__uint_as_float(r[6]), __uint_as_float(r[7])), c2, pack2(n1.z, n1.w));
+                    ex2_mufu2_n(x);
+                    acc_a = add2(acc_a, x[0]); acc_b = add2(acc_b, x[1]);
+                    acc_a = add2(acc_a, x[2]); acc_b = add2(acc_b, x[3]);
                 } else {
 #pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (c0 + e < rows) acc[e & 3] += ex2(fmaf(__uint_as_float(r[e]), scale_log2, neg_lse_s[c0 + e]));
+                    for (int e = 0; e < 8; ++e)
+                        if (c0 + e < col_hi) tail += ex2(fmaf(__uint_as_float(r[e]), scale_log2, neg_lse_s[c0 + e]));
+                }
+            };
+            if (col_lo < col_hi) {
+                uint32_t ra[8], rb[8];
+                tmem_ld8(taddr + col_lo, ra);
+                for (int c0 = col_lo; c0 < col_hi; c0 += 16) {
+                    tmem_wait_ld(ra);
+                    if (c0 + 8 < col_hi) tmem_ld8(taddr + c0 + 8, rb);
+                    unit(ra, c0);
+                    if (c0 + 8 < col_hi) {
+                        tmem_wait_ld(rb);
+                        if (c0 + 16 < col_hi) tmem_ld8(taddr + c0 + 16, ra);
+                        unit(rb, c0 + 8);
+                    }
                 }
             }
             tc_fence_before_sync();
-            mbar_arrive(bar(T_EMPTY + wg));
-            const int j = (tile0 + i) * kTile + w4 * 32 + lane;
-            if (j < N) {
-                const float v = ((acc[0] + acc[1]) + (acc[2] + acc[3])) * inv_m;
-                srow[j] = accumulate ? srow[j] + v : v;
+            mbar_arrive(bar(T_EMPTY + buf));
+            float a0, a1, b0, b1;
+            unpack2(acc_a, a0, a1); unpack2(acc_b, b0, b1);
+            const float sum = ((a0 + a1) + (b0 + b1)) + tail;
+            if (wg > 0) {
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(P_EMPTY + buf), (ub & 1) ^ 1, abort_s, status))) break;
+                part_s[(buf * (kScoreWgs - 1) + wg - 1) * 128 + key] = sum;
+                mbar_arrive(bar(P_FULL + buf));
+            } else {
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(P_FULL + buf), ub & 1, abort_s, status))) break;
+                float v = sum;
+#pragma unroll
+                for (int g = 0; g < kScoreWgs - 1; ++g) v += part_s[(buf * (kScoreWgs - 1) + g) * 128 + key];
+                mbar_arrive(bar(P_EMPTY + buf));
+                v *= inv_m;
+                const int j = (tile0 + i) * kTile + key;
+                if (j < N) srow[j] = accumulate ? srow[j] + v : v;
             }
         }
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 9) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
+    if (warp == kScoreMmaWarp) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
 }
-
 
 // ------------------------------------------------------------------------------------------------------------
 // Attention kernel (Algorithm 1: "Attn(Q, K, V, C)" over one chunk of the prefix, and "SparseAttn" over the
@@ -192,9 +240,12 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
 // SPARSE (SPARSE = true): four producer warps gather the k_eff selected cache rows (then the block's keys) with
 //         16-byte cp.async into the same swizzled layout; the result is the final bf16 output.
 // ------------------------------------------------------------------------------------------------------------
-constexpr int kAttnSlots = 5;                          // ring of K/V tile slots: K(0) V(0) K(1) V(1) ...
+constexpr int kAttnSlotsDense = 5;                     // ring of K/V tile slots: K(0) V(0) K(1) V(1) ...
+constexpr int kAttnSlotsSparse = 4;                    // one slot less: the room holds the gathered rows' offset table
+constexpr int kSparseTableCap = 4096;                  // selected rows whose cache offsets are tabulated in shared memory
 constexpr int kAttnQBytes = 2 * kTileBytes;            // two M-tiles of 128 rows
-constexpr size_t kAttnSmemBytes = 1024 + kAttnQBytes + kAttnSlots * kTileBytes + 512;
+constexpr size_t kAttnSmemBytesDense = 1024 + kAttnQBytes + kAttnSlotsDense * kTileBytes + 512;
+constexpr size_t kAttnSmemBytesSparse = 1024 + kAttnQBytes + kAttnSlotsSparse * kTileBytes + 512 + kSparseTableCap * sizeof(int);
 constexpr float kRescaleThreshold = 8.f;               // log2 units
 
 struct AttnMaps { CUtensorMap q, k, v, kb, vb; };
@@ -206,6 +257,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             float scale_log2, float *__restrict__ ws, __nv_bfloat16 *__restrict__ out, unsigned *status) {
     using namespace ptx;
     constexpr int kMmaWarp = SPARSE ? 12 : 9;
+    constexpr int kAttnSlots = SPARSE ? kAttnSlotsSparse : kAttnSlotsDense;
     const int chunk = blockIdx.x, rg = blockIdx.y, z = blockIdx.z, p = z / kv.H_kv, h = z % kv.H_kv;
     const int N = seq_len_of(kv, p);
     int n_keys, n_cache, j_begin = 0;
@@ -234,6 +286,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
     enum { Q_FULL = 0, FULL = 1, EMPTY = FULL + kAttnSlots, S_FULL = EMPTY + kAttnSlots, P_FULL = S_FULL + 2, O_DONE = P_FULL + 2, N_BARS = O_DONE + 1 };
     uint32_t *tmem_ptr_s = reinterpret_cast<uint32_t *>(bars + N_BARS);
     volatile int *abort_s = reinterpret_cast<volatile int *>(tmem_ptr_s + 1);
+    int *row_tab = reinterpret_cast<int *>(tmem_ptr_s + 4);     // SPARSE: cache offset / 8 of each selected row, -1 = skip
     auto bar = [&](int i) { return smem_u32(bars + i); };
     auto slot_of = [](int L) { return L % kAttnSlots; };
     auto par_of = [](int L) { return (L / kAttnSlots) & 1; };
@@ -248,6 +301,20 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
         fence_mbar_init();
     }
     if (warp == kMmaWarp) { tmem_alloc(smem_u32(tmem_ptr_s), 512); tmem_relinquish(); }
+    // SPARSE: resolve every selected index to a cache row once (shared by the K and V gathers): bounds check,
+    // page-table lookup, offset in 16-byte units.  Budgets beyond the table are resolved on the fly.
+    auto resolve = [&](int t) -> int {
+        const int j = indices[(long long)z * k + t];
+        if (j < 0 || j >= N) {
+            if (status) atomicOr(status, MAGE_DEV_BAD_INDEX);
+            return -1;
+        }
+        const long long off = cache_row_offset(kv, p, h, j, status);
+        return off < 0 ? -1 : (int)(off >> 3);
+    };
+    const bool use_tab = SPARSE && n_cache <= kSparseTableCap;
+    if (use_tab)
+        for (int t = tid; t < n_cache; t += blockDim.x) row_tab[t] = resolve(t);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -302,13 +369,8 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     uint8_t *dst = tile + r * 128 + (((cchunk & 7) ^ (r & 7)) << 4);
                     const __nv_bfloat16 *src = nullptr;
                     if (t < n_cache) {
-                        const int j = indices[(long long)z * k + t];
-                        if (j >= 0 && j < N) {
-                            const long long off = cache_row_offset(kv, p, h, j, status);
-                            if (off >= 0) src = cache + off + cchunk * 8;
-                        } else if (status) {
-                            atomicOr(status, MAGE_DEV_BAD_INDEX);
-                        }
+                        const int o = use_tab ? row_tab[t] : resolve(t);
+                        if (o >= 0) src = cache + ((long long)o << 3) + cchunk * 8;
                     } else if (t < n_keys) {
                         src = blk + ((long long)z * kv.B + (t - n_cache)) * kD + cchunk * 8;
                     }
@@ -402,70 +464,138 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             const uint32_t tS = tmem_base + mt * 128 + lane_off, tO = tmem_base + 256 + mt * 128 + lane_off;
             const int row = w4 * 32 + lane, grow = rg * 256 + mt * kTile + row;
             float m_used = -INFINITY, l = 0.f;
+            float pend_m = 0.f;          // reference the row wants to move to at the start of its next tile
+            bool pending = false;
+            const uint64_t c2 = pack2(scale_log2, scale_log2);
             bool ok = true;
             for (int i = 0; i < n_tiles; ++i) {
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(S_FULL + mt), i & 1, abort_s, status))) { ok = false; break; }
                 tc_fence_after_sync();
                 const int valid = min(kTile, n_keys - i * kTile);
-                float mx = -INFINITY;
+                // Rescale O by f (rows that do not need it pass f = 1): no MMA touches this O between "S(i) complete"
+                // (which implies PV(i-1) complete) and "P(i) ready".
+                auto rescale_o = [&](float f) {
 #pragma unroll
-                for (int c0 = 0; c0 < kTile; c0 += 32) {
-                    uint32_t r[32];
-                    tmem_ld32(tS + c0, r);
-                    tmem_wait_ld();
-                    if (valid == kTile) {
+                    for (int c0 = 0; c0 < kD; c0 += 32) {
+                        uint32_t r[32];
+                        tmem_ld32(tO + c0, r);
+                        tmem_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]));
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (c0 + e < valid) mx = fmaxf(mx, __uint_as_float(r[e]));
+                        for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * f);
+                        tmem_st32(tO + c0, r);
                     }
-                }
-                const float mx_s = mx * scale_log2;
-                if (i == 0) {
-                    m_used = mx_s;
-                } else {
-                    const bool need = mx_s > m_used + kRescaleThreshold;
-                    if (__any_sync(0xffffffffu, need)) {
-                        const float m_new = need ? mx_s : m_used;
-                        const float f = ex2(m_used - m_new);
+                    tmem_wait_st();
+                };
+                bool fast = i > 0 && valid == kTile;
+                if (fast) {
+                    // ---- common case: one sweep over S with the reference maximum carried over from earlier tiles.
+                    // exp2(x - m_used) stays representable as long as x - m_used < 100, so the true maximum is only
+                    // tracked (to move the reference lazily, at the next tile) and checked against that limit.
+                    if (__any_sync(0xffffffffu, pending)) {
+                        const float f = pending ? ex2(m_used - pend_m) : 1.f;
+                        rescale_o(f);
                         l *= f;
+                        if (pending) m_used = pend_m;
+                        pending = false;
+                    }
+                    const uint64_t neg_m2 = pack2(-m_used, -m_used);
+                    uint64_t l2a = pack2(0.f, 0.f), l2b = l2a;
+                    float mx = -INFINITY;
+                    uint32_t pk[64];
+                    auto chunk = [&](const uint32_t (&r)[32], int c) {
 #pragma unroll
-                        for (int c0 = 0; c0 < kD; c0 += 32) {
-                            uint32_t r[32];
-                            tmem_ld32(tO + c0, r);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * f);
-                            tmem_st32(tO + c0, r);
+                        for (int e = 0; e < 16; ++e) {
+                            const uint64_t x2 = fma2(pack2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1])), c2, neg_m2);
+                            float x0, x1;
+                            unpack2(x2, x0, x1);
+                            mx = fmaxf(mx, fmaxf(x0, x1));
+                            const float p0 = ex2(x0), p1 = ex2(x1);
+                            if (e & 1) l2b = add2(l2b, pack2(p0, p1));
+                            else l2a = add2(l2a, pack2(p0, p1));
+                            pk[c * 16 + e] = pack_bf16x2(p0, p1);
                         }
-                        tmem_wait_st();
-                        m_used = m_new;
+                    };
+                    uint32_t ra[32], rb[32];
+                    tmem_ld32(tS, ra);
+                    tmem_wait_ld(ra);
+                    tmem_ld32(tS + 32, rb);
+                    chunk(ra, 0);
+                    tmem_wait_ld(rb);
+                    tmem_ld32(tS + 64, ra);
+                    chunk(rb, 1);
+                    tmem_wait_ld(ra);
+                    tmem_ld32(tS + 96, rb);
+                    chunk(ra, 2);
+                    tmem_wait_ld(rb);
+                    chunk(rb, 3);
+                    if (__any_sync(0xffffffffu, mx > 100.f)) {
+                        fast = false;                     // S is still intact: redo this tile on the careful path
+                    } else {
+                        float a0, a1, b0, b1;
+                        unpack2(l2a, a0, a1);
+                        unpack2(l2b, b0, b1);
+                        l += (a0 + a1) + (b0 + b1);
+                        if (mx > kRescaleThreshold) { pending = true; pend_m = m_used + mx; }
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) tmem_st16(tS + 16 * c, *reinterpret_cast<const uint32_t(*)[16]>(&pk[16 * c]));
                     }
                 }
-                const float neg_m = -m_used;
-                float l0 = 0.f, l1 = 0.f;
+                if (!fast) {
+                    // ---- careful path (first tile, ragged last tile, or a jump of the maximum by more than 2^100):
+                    // find the tile's maximum first, move the reference if it grew, then exponentiate.
+                    float mx = -INFINITY;
 #pragma unroll
-                for (int c0 = 0; c0 < kTile; c0 += 32) {
-                    uint32_t r[32], pk[16];
-                    tmem_ld32(tS + c0, r);
-                    tmem_wait_ld();
+                    for (int c0 = 0; c0 < kTile; c0 += 32) {
+                        uint32_t r[32];
+                        tmem_ld32(tS + c0, r);
+                        tmem_wait_ld();
+                        if (valid == kTile) {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        float p0 = ex2(fmaf(__uint_as_float(r[2 * e]), scale_log2, neg_m));
-                        float p1 = ex2(fmaf(__uint_as_float(r[2 * e + 1]), scale_log2, neg_m));
-                        if (valid != kTile) {
-                            if (c0 + 2 * e >= valid) p0 = 0.f;
-                            if (c0 + 2 * e + 1 >= valid) p1 = 0.f;
+                            for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]));
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 32; ++e)
+                                if (c0 + e < valid) mx = fmaxf(mx, __uint_as_float(r[e]));
                         }
-                        l0 += p0;
-                        l1 += p1;
-                        pk[e] = pack_bf16x2(p0, p1);
                     }
-                    tmem_st16(tS + (c0 >> 1), pk);
+                    float target = mx * scale_log2;
+                    if (pending) target = fmaxf(target, pend_m);
+                    if (i == 0) {
+                        m_used = target;
+                    } else {
+                        const bool need = pending || target > m_used + kRescaleThreshold;
+                        if (__any_sync(0xffffffffu, need)) {
+                            const float m_new = need ? fmaxf(target, m_used) : m_used;
+                            const float f = ex2(m_used - m_new);
+                            rescale_o(f);
+                            l *= f;
+                            m_used = m_new;
+                        }
+                    }
+                    pending = false;
+                    const float neg_m = -m_used;
+                    float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+                    for (int c0 = 0; c0 < kTile; c0 += 32) {
+                        uint32_t r[32], pk[16];
+                        tmem_ld32(tS + c0, r);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            float p0 = ex2(fmaf(__uint_as_float(r[2 * e]), scale_log2, neg_m));
+                            float p1 = ex2(fmaf(__uint_as_float(r[2 * e + 1]), scale_log2, neg_m));
+                            if (valid != kTile) {
+                                if (c0 + 2 * e >= valid) p0 = 0.f;
+                                if (c0 + 2 * e + 1 >= valid) p1 = 0.f;
+                            }
+                            l0 += p0;
+                            l1 += p1;
+                            pk[e] = pack_bf16x2(p0, p1);
+                        }
+                        tmem_st16(tS + (c0 >> 1), pk);
+                    }
+                    l += l0 + l1;
                 }
-                l += l0 + l1;
                 tmem_wait_st();
                 if (!SPARSE && valid != kTile && mt == 0) {
                     // Last tile of the prefix: cache rows past the end may hold anything (even NaN patterns), and

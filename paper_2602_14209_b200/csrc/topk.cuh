@@ -13,8 +13,8 @@ __device__ __forceinline__ unsigned float_order_key(float f) {
 }
 
 // One CTA per (problem, KV head).
-//  1. four 8-bit radix passes over the keys find the k_eff-th largest key T and how many entries equal to T
-//     are still needed (histograms in shared memory, warp-aggregated atomics);
+//  1. a min/max pass finds the keys' common leading bits; radix passes of up to 8 bits over the remaining bits
+//     find the k_eff-th largest key T and how many entries equal to T are still needed (shared-memory histograms);
 //  2. one ordered pass emits every position with key > T and the first `need_eq` positions with key == T,
 //     placed by a block-wide prefix sum, so the output is ascending and ties go to the smaller position.
 __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *__restrict__ scores,
@@ -39,49 +39,91 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *__restr
         return;
     }
 
-    unsigned prefix = 0, mask = 0, need = (unsigned)k_eff;
-    for (int pass = 0; pass < 4; ++pass) {
-        const int shift = 24 - 8 * pass;
-        if (tid < 256) hist[tid] = 0;
-        __syncthreads();
-        for (int j0 = 0; j0 < N; j0 += kTopkThreads) {
-            const int j = j0 + tid;
-            unsigned key = 0;
-            bool valid = j < N;
-            if (valid) { key = float_order_key(s[j]); valid = (key & mask) == prefix; }
-            const unsigned digit = (key >> shift) & 255u;
-            const unsigned peers = __match_any_sync(0xffffffffu, valid ? digit : 256u + lane);
-            if (valid && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
+    const bool vec_ok = (reinterpret_cast<uintptr_t>(s) & 15) == 0;
+    // Visit the row 8 elements per thread and iteration, all loads issued before any is used.
+    auto for_each8 = [&](auto &&body) {
+        for (int base = 0; base < N; base += kTopkThreads * 8) {
+            float v[8];
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int j = base + half * kTopkThreads * 4 + tid * 4;
+                if (vec_ok && j + 3 < N) {
+                    const float4 f = *reinterpret_cast<const float4 *>(s + j);
+                    v[half * 4 + 0] = f.x; v[half * 4 + 1] = f.y; v[half * 4 + 2] = f.z; v[half * 4 + 3] = f.w;
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) v[half * 4 + e] = j + e < N ? s[j + e] : 0.f;
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int j = base + (e >> 2) * kTopkThreads * 4 + tid * 4 + (e & 3);
+                if (j < N) body(float_order_key(v[e]));
+            }
         }
-        __syncthreads();
-        // suffix[t] = number of candidates whose digit is >= t
-        if (tid < 256) suffix[tid] = hist[tid];
-        if (tid == 0) suffix[256] = 0;
-        __syncthreads();
-        for (int off = 1; off < 256; off <<= 1) {
-            unsigned add = 0;
-            if (tid < 256 && tid + off < 256) add = suffix[tid + off];
+    };
+
+    // Pass 0: smallest and largest key.  Their common leading bits need no radix pass (block scores of one head
+    // usually share sign, exponent and a few mantissa bits), and a constant row is decided here.
+    unsigned kmin = 0xffffffffu, kmax = 0u;
+    for_each8([&](unsigned key) { kmin = min(kmin, key); kmax = max(kmax, key); });
+    kmin = __reduce_min_sync(0xffffffffu, kmin);
+    kmax = __reduce_max_sync(0xffffffffu, kmax);
+    if (lane == 0) { warp_tot[warp] = kmin; hist[warp] = kmax; }
+    __syncthreads();
+    if (warp == 0) {
+        kmin = __reduce_min_sync(0xffffffffu, warp_tot[lane]);
+        kmax = __reduce_max_sync(0xffffffffu, hist[lane]);
+        if (lane == 0) { suffix[0] = kmin; suffix[1] = kmax; }
+    }
+    __syncthreads();
+    kmin = suffix[0];
+    kmax = suffix[1];
+    __syncthreads();
+
+    unsigned prefix = kmax, mask = 0xffffffffu, need = (unsigned)k_eff;
+    if (kmin != kmax) {
+        int hi = 31 - __clz(kmin ^ kmax);                 // highest bit in which any two keys differ
+        mask = hi == 31 ? 0u : ~((2u << hi) - 1u);
+        prefix = kmax & mask;
+        // Radix passes of up to 8 bits from there down.  Only keys that still match the prefix touch the
+        // histogram, so after the first pass the shared-memory atomics are few.
+        while (hi >= 0) {
+            const int lo = hi >= 7 ? hi - 7 : 0;
+            const unsigned dmask = (1u << (hi - lo + 1)) - 1u;
+            if (tid < 256) hist[tid] = 0;
             __syncthreads();
-            if (tid < 256) suffix[tid] += add;
+            for_each8([&](unsigned key) {
+                if ((key & mask) == prefix) atomicAdd(&hist[(key >> lo) & dmask], 1u);
+            });
             __syncthreads();
+            // suffix[t] = number of candidates whose digit is >= t
+            if (tid < 256) suffix[tid] = hist[tid];
+            if (tid == 0) suffix[256] = 0;
+            __syncthreads();
+            for (int off = 1; off < 256; off <<= 1) {
+                unsigned add = 0;
+                if (tid < 256 && tid + off < 256) add = suffix[tid + off];
+                __syncthreads();
+                if (tid < 256) suffix[tid] += add;
+                __syncthreads();
+            }
+            if (tid < 256 && suffix[tid] >= need && suffix[tid + 1] < need) {
+                sel_digit = tid;
+                sel_need = need - suffix[tid + 1];
+            }
+            __syncthreads();
+            prefix |= sel_digit << lo;
+            mask |= dmask << lo;
+            need = sel_need;
+            __syncthreads();
+            hi = lo - 1;
         }
-        if (tid < 256 && suffix[tid] >= need && suffix[tid + 1] < need) {
-            sel_digit = tid;
-            sel_need = need - suffix[tid + 1];
-        }
-        __syncthreads();
-        prefix |= sel_digit << shift;
-        mask |= 255u << shift;
-        need = sel_need;
-        __syncthreads();
     }
     const unsigned T = prefix, need_eq = need;
 
-    const bool vec_ok = (reinterpret_cast<uintptr_t>(s) & 15) == 0;
     unsigned run_gt = 0, run_eq = 0;
-    for (int base = 0; base < N; base += kTopkThreads * 4) {
-        const int j_first = base + tid * 4;
-        float v[4];
+    auto load4 = [&](int j_first, float (&v)[4]) {
         if (vec_ok && j_first + 3 < N) {
             const float4 f = *reinterpret_cast<const float4 *>(s + j_first);
             v[0] = f.x; v[1] = f.y; v[2] = f.z; v[3] = f.w;
@@ -89,6 +131,13 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *__restr
 #pragma unroll
             for (int e = 0; e < 4; ++e) v[e] = j_first + e < N ? s[j_first + e] : 0.f;
         }
+    };
+    float nxt[4];
+    load4(tid * 4, nxt);
+    for (int base = 0; base < N; base += kTopkThreads * 4) {
+        const int j_first = base + tid * 4;
+        float v[4] = {nxt[0], nxt[1], nxt[2], nxt[3]};
+        if (base + kTopkThreads * 4 < N) load4(j_first + kTopkThreads * 4, nxt);     // prefetch the next chunk
         unsigned gt = 0, eq = 0, is_gt = 0, is_eq = 0;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
