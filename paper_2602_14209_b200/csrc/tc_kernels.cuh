@@ -283,7 +283,8 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *q_s = base, *kv_s = base + kAttnQBytes;
     uint64_t *bars = reinterpret_cast<uint64_t *>(kv_s + kAttnSlots * kTileBytes);
-    enum { Q_FULL = 0, FULL = 1, EMPTY = FULL + kAttnSlots, S_FULL = EMPTY + kAttnSlots, P_FULL = S_FULL + 2, O_DONE = P_FULL + 2, N_BARS = O_DONE + 1 };
+    enum { Q_FULL = 0, FULL = 1, EMPTY = FULL + kAttnSlots, S_FULL = EMPTY + kAttnSlots, P_HALF = S_FULL + 2, P_FULL = P_HALF + 2,
+           PVH_DONE = P_FULL + 2, O_DONE = PVH_DONE + 2, N_BARS = O_DONE + 1 };
     uint32_t *tmem_ptr_s = reinterpret_cast<uint32_t *>(bars + N_BARS);
     volatile int *abort_s = reinterpret_cast<volatile int *>(tmem_ptr_s + 1);
     int *row_tab = reinterpret_cast<int *>(tmem_ptr_s + 4);     // SPARSE: cache offset / 8 of each selected row, -1 = skip
@@ -296,7 +297,12 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
         *abort_s = 0;
         mbar_init(bar(Q_FULL), 1);
         for (int s = 0; s < kAttnSlots; ++s) { mbar_init(bar(FULL + s), SPARSE ? 128 : 1); mbar_init(bar(EMPTY + s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(bar(S_FULL + b), 1); mbar_init(bar(P_FULL + b), 128); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar(S_FULL + b), 1);
+            mbar_init(bar(P_HALF + b), 128);
+            mbar_init(bar(P_FULL + b), 128);
+            mbar_init(bar(PVH_DONE + b), 1);
+        }
         mbar_init(bar(O_DONE), 1);
         fence_mbar_init();
     }
@@ -414,10 +420,10 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     umma_ss(tmem_base + mt * 128, a, b, idesc_qk, ks > 0);
                 }
             };
-            auto pv = [&](int i, int mt) {
+            auto pv = [&](int i, int mt, int half) {  // half 0: keys 0-63 of the tile, half 1: keys 64-127
                 const uint32_t v_addr = smem_u32(kv_s + slot_of(2 * i + 1) * kTileBytes);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {      // 16 keys per step: 16 rows of 128 bytes in each d-half
+                for (int ks = half * 4; ks < half * 4 + 4; ++ks) {      // 16 keys per step: 16 rows of 128 bytes in each d-half
                     const uint64_t b = smem_desc_sw128(v_addr + ks * 2048, kHalfBytes, 1024);
                     umma_ts(tmem_base + 256 + mt * 128, tmem_base + mt * 128 + ks * 8, b, idesc_pv, (i > 0 || ks > 0) ? 1u : 0u);
                 }
@@ -434,9 +440,13 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             for (int i = 0; ok && i < n_tiles; ++i) {
                 const bool more = i + 1 < n_tiles;
                 if (!mbar_wait(bar(FULL + slot_of(2 * i + 1)), par_of(2 * i + 1), abort_s, status)) break;
+                if (!mbar_wait(bar(P_HALF + 0), i & 1, abort_s, status)) break;
+                tc_fence_after_sync();
+                pv(i, 0, 0);
+                umma_commit(bar(PVH_DONE + 0));
                 if (!mbar_wait(bar(P_FULL + 0), i & 1, abort_s, status)) break;
                 tc_fence_after_sync();
-                pv(i, 0);
+                pv(i, 0, 1);
                 if (more) {
                     if (!mbar_wait(bar(FULL + slot_of(2 * i + 2)), par_of(2 * i + 2), abort_s, status)) break;
                     tc_fence_after_sync();
@@ -444,9 +454,13 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     umma_commit(bar(S_FULL + 0));
                 }
                 if (n_mt == 2) {
+                    if (!mbar_wait(bar(P_HALF + 1), i & 1, abort_s, status)) break;
+                    tc_fence_after_sync();
+                    pv(i, 1, 0);
+                    umma_commit(bar(PVH_DONE + 1));
                     if (!mbar_wait(bar(P_FULL + 1), i & 1, abort_s, status)) break;
                     tc_fence_after_sync();
-                    pv(i, 1);
+                    pv(i, 1, 1);
                 }
                 umma_commit(bar(EMPTY + slot_of(2 * i + 1)));
                 if (more) {
@@ -486,7 +500,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     }
                     tmem_wait_st();
                 };
-                bool fast = i > 0 && valid == kTile;
+                bool fast = i > 0 && valid == kTile, half_done = false;
                 if (fast) {
                     // ---- common case: one sweep over S with the reference maximum carried over from earlier tiles.
                     // exp2(x - m_used) stays representable as long as x - m_used < 100, so the true maximum is only
@@ -498,11 +512,11 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                         if (pending) m_used = pend_m;
                         pending = false;
                     }
-                    const uint64_t neg_m2 = pack2(-m_used, -m_used);
+                    uint64_t neg_m2 = pack2(-m_used, -m_used);
                     uint64_t l2a = pack2(0.f, 0.f), l2b = l2a;
                     float mx = -INFINITY;
-                    uint32_t pk[64];
-                    auto chunk = [&](const uint32_t (&r)[32], int c) {
+                    // 32 columns of S -> 16 packed bf16 pairs of P, the row sum and the running maximum of x
+                    auto chunk = [&](const uint32_t (&r)[32], uint32_t (&pk)[16]) {
 #pragma unroll
                         for (int e = 0; e < 16; ++e) {
                             const uint64_t x2 = fma2(pack2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1])), c2, neg_m2);
@@ -512,32 +526,83 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                             const float p0 = ex2(x0), p1 = ex2(x1);
                             if (e & 1) l2b = add2(l2b, pack2(p0, p1));
                             else l2a = add2(l2a, pack2(p0, p1));
-                            pk[c * 16 + e] = pack_bf16x2(p0, p1);
+                            pk[e] = pack_bf16x2(p0, p1);
                         }
                     };
-                    uint32_t ra[32], rb[32];
+                    uint32_t ra[32], rb[32], pa[16], pb[16];
+                    // first half of the tile (keys 0-63): nothing is stored before its maximum has been checked, so S
+                    // is still whole if the tile has to be redone on the careful path
                     tmem_ld32(tS, ra);
                     tmem_wait_ld(ra);
                     tmem_ld32(tS + 32, rb);
-                    chunk(ra, 0);
+                    chunk(ra, pa);
                     tmem_wait_ld(rb);
                     tmem_ld32(tS + 64, ra);
-                    chunk(rb, 1);
-                    tmem_wait_ld(ra);
-                    tmem_ld32(tS + 96, rb);
-                    chunk(ra, 2);
-                    tmem_wait_ld(rb);
-                    chunk(rb, 3);
+                    chunk(rb, pb);
                     if (__any_sync(0xffffffffu, mx > 100.f)) {
-                        fast = false;                     // S is still intact: redo this tile on the careful path
+                        tmem_wait_ld(ra);
+                        fast = false;
                     } else {
+                        tmem_st16(tS, pa);
+                        tmem_st16(tS + 16, pb);
+                        tmem_wait_ld(ra);
+                        tmem_ld32(tS + 96, rb);
+                        tmem_wait_st();
+                        tc_fence_before_sync();
+                        mbar_arrive(bar(P_HALF + mt));         // the PV MMA may start on keys 0-63
+                        half_done = true;
+                        // second half (keys 64-127): its P lands on S columns 32-63, already consumed; its own S
+                        // columns 64-127 are never overwritten
+                        const float mx_first = mx;
+                        mx = -INFINITY;
+                        chunk(ra, pa);
+                        tmem_wait_ld(rb);
+                        chunk(rb, pb);
+                        if (__any_sync(0xffffffffu, mx > 100.f)) {
+                            // A jump of more than 2^100 inside the tile (never seen in practice; kept for correctness):
+                            // wait until the first half's PV has been accumulated, move the reference, redo keys 64-127.
+                            if (!__all_sync(0xffffffffu, mbar_wait(bar(PVH_DONE + mt), i & 1, abort_s, status))) { ok = false; break; }
+                            tc_fence_after_sync();
+                            float a0, a1, b0, b1;
+                            unpack2(l2a, a0, a1);
+                            unpack2(l2b, b0, b1);
+                            // l2a/l2b hold first-half terms (valid) and second-half terms (overflowed): recompute both
+                            const float m_new = fmaxf(m_used, m_used + fmaxf(mx, mx_first));
+                            const float f = ex2(m_used - m_new);
+                            rescale_o(f);
+                            l *= f;
+                            float l_first = 0.f;           // first-half row sum, recomputed from the stored bf16 P
+#pragma unroll
+                            for (int c0 = 0; c0 < 32; c0 += 16) {
+                                uint32_t pr[16];
+                                tmem_ld16(tS + c0, pr);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int e = 0; e < 16; ++e) l_first += __uint_as_float(pr[e] << 16) + __uint_as_float(pr[e] & 0xffff0000u);
+                            }
+                            l += l_first * f;
+                            m_used = m_new;
+                            neg_m2 = pack2(-m_used, -m_used);
+                            l2a = pack2(0.f, 0.f);
+                            l2b = l2a;
+                            mx = -INFINITY;
+                            tmem_ld32(tS + 64, ra);
+                            tmem_wait_ld(ra);
+                            tmem_ld32(tS + 96, rb);
+                            chunk(ra, pa);
+                            tmem_wait_ld(rb);
+                            chunk(rb, pb);
+                            mx = 0.f;
+                        } else {
+                            mx = fmaxf(mx, mx_first);
+                        }
                         float a0, a1, b0, b1;
                         unpack2(l2a, a0, a1);
                         unpack2(l2b, b0, b1);
                         l += (a0 + a1) + (b0 + b1);
                         if (mx > kRescaleThreshold) { pending = true; pend_m = m_used + mx; }
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) tmem_st16(tS + 16 * c, *reinterpret_cast<const uint32_t(*)[16]>(&pk[16 * c]));
+                        tmem_st16(tS + 32, pa);
+                        tmem_st16(tS + 48, pb);
                     }
                 }
                 if (!fast) {
@@ -613,6 +678,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     fence_proxy_async();
                 }
                 tc_fence_before_sync();
+                if (!half_done) mbar_arrive(bar(P_HALF + mt));
                 mbar_arrive(bar(P_FULL + mt));
             }
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(O_DONE), 0, abort_s, status));

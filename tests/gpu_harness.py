@@ -60,7 +60,8 @@ def check_topk_band(score_ref, idx_gpu, k, N):
     return k_eff - int(chosen[ref_set].sum())                      # positions that differ (all inside the band)
 
 
-def check_problem(oracle, batch, res, w, p, heads=None, check_scores=True, sparse_steps=None):
+def check_problem(oracle, batch, res, w, p, heads=None, check_scores=True, sparse_steps=None, check_topk=True,
+                  o_max_abs=O_MAX_ABS):
     """Compare problem p of a GPU run with the oracle on the listed KV heads (default: all).  Returns diagnostics."""
     G, B, k = w.G, w.B, res["k"]
     N = int(batch["seq_lens"][p])
@@ -76,8 +77,8 @@ def check_problem(oracle, batch, res, w, p, heads=None, check_scores=True, spars
         err = np.abs(res["outs"][0][p, qs] - O)
         assert np.isfinite(res["outs"][0][p, qs]).all()
         diag["o_max"], diag["o_mean"] = max(diag["o_max"], err.max()), max(diag["o_mean"], err.mean())
-        assert err.max() <= O_MAX_ABS and err.mean() <= O_MEAN_ABS, (p, h, err.max(), err.mean())
-        if N > 0:
+        assert err.max() <= o_max_abs and err.mean() <= O_MEAN_ABS, (p, h, err.max(), err.mean())
+        if N > 0 and check_topk:
             sc = oracle.block_score(f(batch["q"][0, p, qs]), Kc)[0]
             got = res["scores"][p, h, :N].astype(np.float64)
             rel = np.max(np.abs(got - sc) / sc)
@@ -86,7 +87,7 @@ def check_problem(oracle, batch, res, w, p, heads=None, check_scores=True, spars
                 assert rel <= SCORE_REL, (p, h, rel)
             assert (res["scores"][p, h, N:] == -1.0).all(), "scores beyond N_p were written"
             diag["band_swaps"] += check_topk_band(sc, res["indices"][p, h], k, N)
-        else:
+        elif N == 0:
             assert (res["indices"][p, h] == -1).all()
         k_eff = int(res["k_eff"][p])
         for t in (range(1, T) if sparse_steps is None else sparse_steps):
@@ -96,6 +97,6 @@ def check_problem(oracle, batch, res, w, p, heads=None, check_scores=True, spars
             e = np.abs(res["outs"][t][p, qs] - Os)
             assert np.isfinite(res["outs"][t][p, qs]).all()
             diag["sp_max"], diag["sp_mean"] = max(diag["sp_max"], e.max()), max(diag["sp_mean"], e.mean())
-            assert e.max() <= O_MAX_ABS and e.mean() <= O_MEAN_ABS, (p, h, t, e.max(), e.mean())
+            assert e.max() <= o_max_abs and e.mean() <= O_MEAN_ABS, (p, h, t, e.max(), e.mean())
     assert res["status"] == 0
     return diag

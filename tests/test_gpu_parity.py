@@ -135,3 +135,24 @@ def test_bad_indices_and_pages_are_flagged_not_dereferenced():
     torch.cuda.synchronize()
     assert int(ba.status.item()) & mb.DEV_BAD_PAGE
     assert torch.isfinite(ba.out.float()).all()
+
+
+@pytest.mark.parametrize("flags", IMPLS)
+def test_logit_jumps_beyond_the_lazy_rescale_range(oracle_mod, flags):
+    """Keys whose logit exceeds everything seen before by far more than 2^100: the running reference of the online
+    softmax has to move inside a tile (first half and second half) without losing the terms accumulated so far."""
+    w = W.Workload("jumps", H_q=8, H_kv=2, N=1024, B=32, k=64, T=2, n_heavy=8, seed=12)
+    batch = W.make_batch(w, device="cuda")
+    batch["q"][..., 0] = 16.0
+    batch["kc"][..., 0] = 0.0
+    batch["kb"][..., 0] = 0.0
+    for j, val in ((300, 64.0), (450, 144.0), (700, 256.0)):      # tile 2 first half, tile 3 second half, tile 5 first half
+        batch["kc"][:, 0, j, 0] = val
+    batch["kc"][:, 1, 20, 0] = 192.0                               # head 1: the big key sits in the very first tile
+    batch["kc"][:, 1, 1000, 0] = 200.0                             # ... and a moderate rise (no overflow) near the end
+    res = H.run_gpu_block(batch, w, flags=flags)
+    # A row that one key dominates, met while the reference lags behind (rise between 2^8 and 2^100), carries that
+    # key's bf16 rounding of P (relative 2^-9) into O: |err| <= 2^-9 * max|V| + bf16 output rounding.  Hence 2e-2 here.
+    H.check_problem(oracle_mod, batch, res, w, 0, check_topk=False, o_max_abs=2e-2)
+    # the dominant key takes (almost) all of the probability mass of every row
+    assert abs(res["scores"][0, 0, 700] - 1.0) < 1e-5 and res["scores"][0, 0, :700].max() < 1e-30
