@@ -346,12 +346,12 @@ def main():
     roofline["hbm_view"] = {"achieved_gbs": sf["s1_attn_bytes"] / attn_avg_ms / 1e6, "peak_gbs": peaks["hbm_gbs"],
                             "frac_of_measured": sf["s1_attn_bytes"] / attn_avg_ms / 1e6 / peaks["hbm_gbs"],
                             "frac_of_8tbs": sf["s1_attn_bytes"] / attn_avg_ms / 1e6 / 8000.0}
-    prof = os.path.join(ROOT, "profiles", "traffic.json")
+    prof = os.path.join(ROOT, "profiles", "traffic.txt")       # ncu-measured DRAM bytes per launch (see the file's header)
     if os.path.exists(prof):
-        try:
-            roofline["traffic"] = json.load(open(prof)).get("simt" if args.simt else "default", {}).get(w.name)
-        except Exception:
-            pass
+        for ln in open(prof):
+            f = ln.split()
+            if len(f) == 3 and not ln.startswith("#") and f[0] == ("simt" if args.simt else "default") and f[1] == w.name:
+                roofline["traffic"] = int(f[2])
 
     cpu_baseline = None
     if not args.no_cpu_baseline:
