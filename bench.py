@@ -325,6 +325,38 @@ def main():
             "hbm_roofline_ms_block_at_8tbs": (sf["s1_bytes"] + (T - 1) * sf["s3_bytes"]) / 8e9,
         }
         del flush
+        # The same block issued layer by layer, as a model would (config 3 "timed back-to-back"): one exact_select, one
+        # top-k (select stream) and T-1 sparse launches per layer; plain launches, and replayed from a CUDA graph.
+        if not w.page_size and w.P > 1:
+            from paper_2602_14209_b200.pipeline import LayerwiseBlock
+            lw = LayerwiseBlock(batch["kc"], batch["vc"], w.H_q, w.B, w.k, batch["seq_lens"])
+            for _ in range(2):
+                lw.run_block(q_d, kb_d, vb_d, outs)
+            torch.cuda.synchronize()
+            reps = 5
+            a.record()
+            for _ in range(reps):
+                lw.run_block(q_d, kb_d, vb_d, outs)
+            b.record(); torch.cuda.synchronize()
+            stages["layerwise_ms_per_block"] = a.elapsed_time(b) / reps
+            try:
+                g = torch.cuda.CUDAGraph()
+                cap = torch.cuda.Stream()
+                cap.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(cap):
+                    with torch.cuda.graph(g, stream=cap):
+                        lw.run_block(q_d, kb_d, vb_d, outs)
+                torch.cuda.current_stream().wait_stream(cap)
+                g.replay(); torch.cuda.synchronize()
+                a.record()
+                for _ in range(reps):
+                    g.replay()
+                b.record(); torch.cuda.synchronize()
+                stages["layerwise_cuda_graph_ms_per_block"] = a.elapsed_time(b) / reps
+            except Exception as e:      # capture is an optimisation of the launch path only
+                stages["layerwise_cuda_graph_ms_per_block"] = None
+                stages["layerwise_cuda_graph_error"] = str(e)[:200]
+            stages["layerwise_dev_status"] = int(lw.status.item())
 
     if rank != 0:
         if world > 1:

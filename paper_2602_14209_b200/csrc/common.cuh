@@ -55,7 +55,11 @@ struct Plan {
     size_t off_part_o;       // float [P*H_kv][n_chunks+1][Mw][128]   unnormalised partial outputs
     size_t off_part_ml;      // float [P*H_kv][n_chunks+1][Mw][2]     (m, l) in the log2 domain
     size_t off_neg_lse;      // float [P*H_kv][Mw]                    -log2-sum-exp over the prefix, per row
-    size_t total_bytes;
+    int sparse_split_max;    // most CTAs that may share one KV head's selected keys in the reuse step
+    size_t off_sparse_o;     // float [P*H_kv][sparse_split_max][Mw][128]  partial outputs of a split reuse step
+    size_t off_sparse_ml;    // float [P*H_kv][sparse_split_max][Mw][2]
+    size_t total_bytes;      // whole workspace; exact_bytes covers what mage_exact_select touches
+    size_t exact_bytes;
 };
 
 }  // namespace mage

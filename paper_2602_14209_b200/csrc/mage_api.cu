@@ -2,6 +2,7 @@
 #include <algorithm>
 #include <atomic>
 #include <cstdio>
+#include <mutex>
 
 #include "common.cuh"
 #include "simt_kernels.cuh"
@@ -46,16 +47,21 @@ static KvView make_view(const mage_kv_t *kv) {
     return v;
 }
 
-// Split of the prefix for the exact pass: enough (head, chunk) items to fill the 148 SMs a few times over,
-// chunks of at least 1024 keys and a multiple of 128 keys.  Pure function of the description.
-static Plan make_plan(const mage_kv_t *kv) {
+// Split of the prefix for the exact pass into chunks of whole 128-key tiles.  Large jobs get about 12 waves of CTAs
+// over the 148 SMs (good balance, partial results stay a few percent of the K/V traffic); small jobs get one wave
+// with at least ~32 tiles per CTA, because every extra chunk costs a CTA prologue and a row in the merge.
+// Pure function of the description.
+static Plan make_plan(const mage_kv_t *kv, int k_max = 0) {
     Plan pl;
     pl.M = kv->H_q / kv->H_kv * kv->B;
     pl.Mw = (int)align_up(pl.M, 128);
     const int64_t heads = (int64_t)kv->P * kv->H_kv;
-    int64_t want = (1776 + heads - 1) / heads;
-    const int64_t max_chunks = kv->N_max > 0 ? (kv->N_max + 1023) / 1024 : 1;
-    if (want > max_chunks) want = max_chunks;
+    const int64_t tiles_head = kv->N_max > 0 ? (kv->N_max + 127) / 128 : 1;
+    int64_t waves = heads * tiles_head / (148 * 32);
+    if (waves < 1) waves = 1;
+    if (waves > 12) waves = 12;
+    int64_t want = 148 * waves / heads - 1;               // the block's own keys take one more item per head
+    if (want > tiles_head) want = tiles_head;
     if (want < 1) want = 1;
     int64_t len = kv->N_max > 0 ? (kv->N_max + want - 1) / want : 128;
     len = (int64_t)align_up((size_t)len, 128);
@@ -66,6 +72,14 @@ static Plan make_plan(const mage_kv_t *kv) {
     pl.off_part_o = off;  off += items * pl.Mw * kD;
     pl.off_part_ml = off; off += items * pl.Mw * 2;
     pl.off_neg_lse = off; off += (size_t)heads * pl.Mw;
+    pl.exact_bytes = align_up(off * sizeof(float), 256);
+    // reuse step: when a launch has few (head, row-group) pairs, the selected keys of one head are split over several
+    // CTAs whose partial results are merged by a second small kernel; room for that, sized by the largest budget
+    off = pl.exact_bytes / sizeof(float);
+    const int tiles_max = k_max > 0 ? (k_max + kv->B + 127) / 128 : 0;
+    pl.sparse_split_max = tiles_max < 32 ? tiles_max : 32;
+    pl.off_sparse_o = off;  off += (size_t)heads * pl.sparse_split_max * pl.Mw * kD;
+    pl.off_sparse_ml = off; off += (size_t)heads * pl.sparse_split_max * pl.Mw * 2;
     pl.total_bytes = align_up(off * sizeof(float), 256);
     return pl;
 }
@@ -80,10 +94,27 @@ static mage_status launch_check() {
     return MAGE_OK;
 }
 
-template <typename K>
-static mage_status opt_in_smem(K kernel, size_t bytes) {
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess ? MAGE_OK : MAGE_ERR_CUDA;
+// Raise a kernel's dynamic shared memory limit; done once per kernel and device, remembered afterwards.
+static mage_status opt_in_smem_impl(const void *kernel, size_t bytes) {
+    static std::mutex mu;
+    static const void *seen[32];
+    static unsigned long long seen_devs[32];
+    static int n_seen = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MAGE_ERR_CUDA;
+    const unsigned long long bit = 1ull << (dev & 63);
+    std::lock_guard<std::mutex> lock(mu);
+    int slot = -1;
+    for (int i = 0; i < n_seen; ++i)
+        if (seen[i] == kernel) slot = i;
+    if (slot >= 0 && (seen_devs[slot] & bit)) return MAGE_OK;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) return MAGE_ERR_CUDA;
+    if (slot < 0 && n_seen < 32) { slot = n_seen++; seen[slot] = kernel; seen_devs[slot] = 0; }
+    if (slot >= 0) seen_devs[slot] |= bit;
+    return MAGE_OK;
 }
+template <typename K>
+static mage_status opt_in_smem(K kernel, size_t bytes) { return opt_in_smem_impl(reinterpret_cast<const void *>(kernel), bytes); }
 
 static mage_status exact_select_simt(const mage_kv_t *kv, const KvView &view, const Plan &plan, const __nv_bfloat16 *q,
                                      const __nv_bfloat16 *k_blk, const __nv_bfloat16 *v_blk, float sm_scale,
@@ -145,17 +176,33 @@ static mage_status exact_select_simt(const mage_kv_t *kv, const KvView &view, co
 
 static mage_status sparse_simt(const mage_kv_t *kv, const KvView &view, const Plan &plan, const __nv_bfloat16 *q,
                                const __nv_bfloat16 *k_blk, const __nv_bfloat16 *v_blk, const int *indices,
-                               const int *k_eff, int k, float sm_scale, __nv_bfloat16 *out, unsigned *dev_status,
-                               cudaStream_t st) {
+                               const int *k_eff, int k, float sm_scale, __nv_bfloat16 *out, float *ws, bool ws_ok,
+                               unsigned *dev_status, cudaStream_t st) {
     using namespace simt;
     if (!(kv->flags & MAGE_FLAG_SIMT_KERNELS) && tc::encode_fn() != nullptr) {
         tc::AttnMaps maps;
         auto kern_tc = tc::attn_kernel<true>;
         if (tc::make_rows_map(&maps.q, q, (long long)kv->P * kv->H_q * kv->B) && opt_in_smem(kern_tc, tc::kAttnSmemBytesSparse) == MAGE_OK) {
             maps.k = maps.v = maps.kb = maps.vb = maps.q;     // unused by the gather producers
-            dim3 tgrid(1, (view.M + 255) / 256, kv->P * kv->H_kv);
-            kern_tc<<<tgrid, 416, tc::kAttnSmemBytesSparse, st>>>(maps, view, plan, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, nullptr, out, dev_status);
-            return launch_check();
+            const int n_rg = (view.M + 255) / 256, heads = kv->P * kv->H_kv;
+            // few (head, row-group) pairs in the launch: split each head's keys over several CTAs and merge
+            int n_split = 1;
+            if (ws_ok && plan.sparse_split_max > 1) {
+                n_split = 148 / (heads * n_rg);
+                const int tiles = (k + kv->B + 127) / 128;
+                if (n_split > tiles) n_split = tiles;
+                if (n_split > plan.sparse_split_max) n_split = plan.sparse_split_max;
+                if (n_split < 1) n_split = 1;
+            }
+            dim3 tgrid(n_split, n_rg, heads);
+            kern_tc<<<tgrid, 416, tc::kAttnSmemBytesSparse, st>>>(maps, view, plan, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, ws, out, dev_status);
+            if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+            if (n_split > 1) {
+                const int rows_total = heads * view.M;
+                tc::sparse_combine_kernel<<<(rows_total + 3) / 4, 128, 0, st>>>(view, plan, n_split, k, k_eff, ws, out);
+                return launch_check();
+            }
+            return MAGE_OK;
         }
     }
     auto kern = attn_kernel<Mode::kSparseFinal>;
@@ -173,7 +220,7 @@ extern "C" {
 
 size_t mage_workspace_bytes(const mage_kv_t *kv, int32_t k_max) {
     if (!valid_kv(kv, nullptr) || k_max < 1) return 0;
-    return make_plan(kv).total_bytes;
+    return make_plan(kv, k_max).total_bytes;
 }
 
 mage_status mage_exact_select_events(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk,
@@ -184,7 +231,7 @@ mage_status mage_exact_select_events(const mage_kv_t *kv, const void *q, const v
     if (!q || !k_blk || !v_blk || !out || !workspace || (kv->N_max > 0 && !scores)) return MAGE_ERR_INVALID_ARG;
     if (!(sm_scale > 0.f) || (reinterpret_cast<uintptr_t>(workspace) & 255)) return MAGE_ERR_INVALID_ARG;
     const Plan plan = make_plan(kv);
-    if (workspace_bytes < plan.total_bytes) return MAGE_ERR_WORKSPACE;
+    if (workspace_bytes < plan.exact_bytes) return MAGE_ERR_WORKSPACE;
     const KvView view = make_view(kv);
     return exact_select_simt(kv, view, plan, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_blk),
                              static_cast<const __nv_bfloat16 *>(v_blk), sm_scale, static_cast<__nv_bfloat16 *>(out), scores,
@@ -214,12 +261,12 @@ mage_status mage_sparse_block_attn(const mage_kv_t *kv, const void *q, const voi
     if (!valid_kv(kv, &why)) return why;
     if (!q || !k_blk || !v_blk || !out || !indices || !k_eff || k < 1) return MAGE_ERR_INVALID_ARG;
     if (!(sm_scale > 0.f)) return MAGE_ERR_INVALID_ARG;
-    (void)workspace; (void)workspace_bytes;
-    const Plan plan = make_plan(kv);
+    const Plan plan = make_plan(kv, k);
     const KvView view = make_view(kv);
+    const bool ws_ok = workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255) && workspace_bytes >= plan.total_bytes;
     return sparse_simt(kv, view, plan, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_blk),
                        static_cast<const __nv_bfloat16 *>(v_blk), indices, k_eff, k, sm_scale, static_cast<__nv_bfloat16 *>(out),
-                       dev_status, static_cast<cudaStream_t>(stream));
+                       static_cast<float *>(workspace), ws_ok, dev_status, static_cast<cudaStream_t>(stream));
 }
 
 // Scratch for mage_exact_select_static.  In host code this name is only a handle for the runtime, not a device
@@ -231,7 +278,7 @@ mage_status mage_exact_select_static(const mage_kv_t *kv, const void *q, const v
                                      float sm_scale, void *out, float *scores, uint32_t *dev_status, void *stream) {
     mage_status why = MAGE_OK;
     if (!valid_kv(kv, &why)) return why;
-    const size_t need = make_plan(kv).total_bytes;
+    const size_t need = make_plan(kv).exact_bytes;
     if (need > (size_t)MAGE_STATIC_SCRATCH_BYTES) {
         std::fprintf(stderr, "libmage: mage_exact_select_static needs %zu bytes of scratch for this description, the built-in "
                              "array holds %u; use mage_exact_select with a caller workspace\n", need, (unsigned)MAGE_STATIC_SCRATCH_BYTES);

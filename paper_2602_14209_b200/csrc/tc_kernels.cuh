@@ -276,6 +276,18 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
         n_cache = min(max(k_eff_arr[p], 0), k);
         n_keys = n_cache + kv.B;
     }
+    // SPARSE with gridDim.x > 1: this CTA takes tiles [tile_lo, tile_lo + n_tiles) of the head's key list and writes
+    // a partial result; key_off shifts the positions in that list.
+    int key_off = 0, blk_shift = n_cache;     // block key number = local position - blk_shift
+    if (SPARSE && gridDim.x > 1) {
+        const int tiles_all = (n_keys + kTile - 1) / kTile, per = (tiles_all + gridDim.x - 1) / gridDim.x;
+        const int tile_lo = chunk * per;
+        if (tile_lo >= tiles_all) return;
+        key_off = tile_lo * kTile;
+        n_keys = min(n_keys - key_off, per * kTile);
+        blk_shift = n_cache - key_off;
+        n_cache = max(0, blk_shift);
+    }
     const int n_tiles = (n_keys + kTile - 1) / kTile;
     const int rows_here = min(256, kv.M - rg * 256), n_mt = rows_here > 128 ? 2 : 1;
 
@@ -310,7 +322,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
     // SPARSE: resolve every selected index to a cache row once (shared by the K and V gathers): bounds check,
     // page-table lookup, offset in 16-byte units.  Budgets beyond the table are resolved on the fly.
     auto resolve = [&](int t) -> int {
-        const int j = indices[(long long)z * k + t];
+        const int j = indices[(long long)z * k + key_off + t];
         if (j < 0 || j >= N) {
             if (status) atomicOr(status, MAGE_DEV_BAD_INDEX);
             return -1;
@@ -362,8 +374,9 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             }
         } else {
             const int pt = tid - 256, cchunk = pt & 15, r0 = pt >> 4;
-            int prev_slot = -1;
+            // Up to three gathers are in flight: the arrival for load L-2 is posted after load L has been issued.
             bool ok = true;
+            int issued = 0;
             for (int L = 0; L < 2 * n_tiles && ok; ++L) {
                 const int i = L >> 1, is_v = L & 1, slot = slot_of(L);
                 if (!mbar_wait(bar(EMPTY + slot), par_of(L) ^ 1, abort_s, status)) { ok = false; break; }
@@ -378,23 +391,30 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                         const int o = use_tab ? row_tab[t] : resolve(t);
                         if (o >= 0) src = cache + ((long long)o << 3) + cchunk * 8;
                     } else if (t < n_keys) {
-                        src = blk + ((long long)z * kv.B + (t - n_cache)) * kD + cchunk * 8;
+                        src = blk + ((long long)z * kv.B + (t - blk_shift)) * kD + cchunk * 8;
                     }
                     if (src) cp_async_16(smem_u32(dst), src);
                     else *reinterpret_cast<uint4 *>(dst) = make_uint4(0, 0, 0, 0);
                 }
                 cp_async_commit();
-                if (prev_slot >= 0) {
+                issued = L + 1;
+                if (L >= 2) {
+                    cp_async_wait<2>();
+                    fence_proxy_async();
+                    mbar_arrive(bar(FULL + slot_of(L - 2)));
+                }
+            }
+            if (ok) {
+                if (issued >= 2) {
                     cp_async_wait<1>();
                     fence_proxy_async();
-                    mbar_arrive(bar(FULL + prev_slot));
+                    mbar_arrive(bar(FULL + slot_of(issued - 2)));
                 }
-                prev_slot = slot;
-            }
-            cp_async_wait<0>();
-            if (ok && prev_slot >= 0) {
+                cp_async_wait<0>();
                 fence_proxy_async();
-                mbar_arrive(bar(FULL + prev_slot));
+                mbar_arrive(bar(FULL + slot_of(issued - 1)));
+            } else {
+                cp_async_wait<0>();
             }
         }
     } else if (warp == kMmaWarp) {
@@ -704,6 +724,25 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                         pml[0] = m_used;
                         pml[1] = l;
                     }
+                } else if (gridDim.x > 1) {
+                    const size_t item = (size_t)z * gridDim.x + chunk;
+                    float *po = ws + plan.off_sparse_o + (item * plan.Mw + grow) * kD;
+#pragma unroll
+                    for (int c0 = 0; c0 < kD; c0 += 32) {
+                        uint32_t r[32];
+                        tmem_ld32(tO + c0, r);
+                        tmem_wait_ld();
+                        if (row_ok) {
+#pragma unroll
+                            for (int e = 0; e < 32; e += 4)
+                                *reinterpret_cast<uint4 *>(po + c0 + e) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
+                        }
+                    }
+                    if (row_ok) {
+                        float *pml = ws + plan.off_sparse_ml + (item * plan.Mw + grow) * 2;
+                        pml[0] = m_used;
+                        pml[1] = l;
+                    }
                 } else {
                     const float inv = 1.f / l;
                     __nv_bfloat16 *po = out + ((long long)(p * kv.H_q + h * kv.G) * kv.B + grow) * kD;
@@ -731,6 +770,34 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
     tc_fence_before_sync();
     __syncthreads();
     if (warp == kMmaWarp) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
+}
+
+// Merge of a reuse step that was split over n_split CTAs per KV head: one warp per query row, fixed order.
+__global__ void __launch_bounds__(128) sparse_combine_kernel(KvView kv, Plan plan, int n_split, int k, const int *__restrict__ k_eff_arr,
+                                                             const float *__restrict__ ws, __nv_bfloat16 *__restrict__ out) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= kv.P * kv.H_kv * kv.M) return;
+    const int z = warp / kv.M, r = warp % kv.M, p = z / kv.H_kv, h = z % kv.H_kv;
+    const int n_keys = min(max(k_eff_arr[p], 0), k) + kv.B;
+    const int tiles_all = (n_keys + kTile - 1) / kTile, per = (tiles_all + n_split - 1) / n_split;
+    const int used = (tiles_all + per - 1) / per;               // splits that had work
+    const float *ml = ws + plan.off_sparse_ml, *po = ws + plan.off_sparse_o;
+    const size_t item0 = (size_t)z * n_split;
+    float m_all = -INFINITY;
+    for (int c = 0; c < used; ++c) m_all = fmaxf(m_all, ml[((item0 + c) * plan.Mw + r) * 2]);
+    float l_all = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c = 0; c < used; ++c) {
+        const float *e = ml + ((item0 + c) * plan.Mw + r) * 2;
+        const float w = exp2f(e[0] - m_all);
+        l_all += e[1] * w;
+        const float4 v = *reinterpret_cast<const float4 *>(po + ((item0 + c) * plan.Mw + r) * kD + lane * 4);
+        acc.x = fmaf(v.x, w, acc.x); acc.y = fmaf(v.y, w, acc.y); acc.z = fmaf(v.z, w, acc.z); acc.w = fmaf(v.w, w, acc.w);
+    }
+    const float inv = 1.f / l_all;
+    __nv_bfloat16 *dst = out + ((long long)(p * kv.H_q + h * kv.G) * kv.B + r) * kD + lane * 4;
+    __nv_bfloat162 a = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), b = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+    *reinterpret_cast<uint2 *>(dst) = make_uint2(*reinterpret_cast<unsigned *>(&a), *reinterpret_cast<unsigned *>(&b));
 }
 
 }  // namespace tc

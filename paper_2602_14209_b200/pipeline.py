@@ -17,16 +17,20 @@ from . import binding as mb
 class BlockAttention:
     """Owns the outputs and scratch of one batch of problems and issues the three library calls."""
 
-    def __init__(self, kv: mb.KVCache, k: int, sm_scale: Optional[float] = None, select_stream: Optional[torch.cuda.Stream] = None):
+    def __init__(self, kv: mb.KVCache, k: int, sm_scale: Optional[float] = None, select_stream: Optional[torch.cuda.Stream] = None,
+                 buffers: Optional[dict] = None):
+        """``buffers`` lets several instances (e.g. one per layer) live in slices of shared tensors: keys out, scores,
+        indices, k_eff, status, workspace; anything missing is allocated here."""
         self.kv, self.k = kv, int(k)
         self.sm_scale = float(kv.d) ** -0.5 if sm_scale is None else float(sm_scale)
         dev = kv.device
-        self.out = torch.empty(kv.P, kv.H_q, kv.B, kv.d, dtype=torch.bfloat16, device=dev)
-        self.scores = torch.zeros(kv.P, kv.H_kv, max(kv.N_max, 1), dtype=torch.float32, device=dev)
-        self.indices = torch.full((kv.P, kv.H_kv, self.k), -1, dtype=torch.int32, device=dev)
-        self.k_eff = torch.zeros(kv.P, dtype=torch.int32, device=dev)
-        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
-        self.workspace = kv.new_workspace(self.k)
+        b = buffers or {}
+        self.out = b["out"] if "out" in b else torch.empty(kv.P, kv.H_q, kv.B, kv.d, dtype=torch.bfloat16, device=dev)
+        self.scores = b["scores"] if "scores" in b else torch.zeros(kv.P, kv.H_kv, max(kv.N_max, 1), dtype=torch.float32, device=dev)
+        self.indices = b["indices"] if "indices" in b else torch.full((kv.P, kv.H_kv, self.k), -1, dtype=torch.int32, device=dev)
+        self.k_eff = b["k_eff"] if "k_eff" in b else torch.zeros(kv.P, dtype=torch.int32, device=dev)
+        self.status = b["status"] if "status" in b else torch.zeros(1, dtype=torch.int32, device=dev)
+        self.workspace = b["workspace"] if "workspace" in b else kv.new_workspace(self.k)
         self.select_stream = select_stream if select_stream is not None else torch.cuda.Stream(device=dev)
         self._scores_ready = torch.cuda.Event()
         self._indices_ready = torch.cuda.Event()
@@ -72,3 +76,46 @@ class BlockAttention:
         for t in range(1, T):
             res.append(self.sparse_step(q_steps[t], kb_steps[t], vb_steps[t], None if outs is None else outs[t]))
         return res
+
+
+class LayerwiseBlock:
+    """One block of Algorithm 1 issued the way a model runs it: layer after layer.
+
+    Step 1 walks the layers on the main stream (``mage_exact_select`` per layer) while each layer's ``mage_topk`` runs
+    on the select stream behind it; one join; then every reuse step walks the layers again with one
+    ``mage_sparse_block_attn`` per layer.  The batched tensors of a multi-layer workload are sliced per layer, so the
+    per-layer calls see P = 1 descriptions of the same memory.
+    """
+
+    def __init__(self, k_cache: torch.Tensor, v_cache: torch.Tensor, H_q: int, B: int, k: int, seq_lens: torch.Tensor):
+        P = k_cache.shape[0]
+        dev = k_cache.device
+        self.select_stream = torch.cuda.Stream(device=dev)
+        self.P, self.k = P, k
+        H_kv, N_max, d = k_cache.shape[1], k_cache.shape[2], k_cache.shape[3]
+        self.out = torch.empty(P, H_q, B, d, dtype=torch.bfloat16, device=dev)
+        self.scores = torch.zeros(P, H_kv, max(N_max, 1), dtype=torch.float32, device=dev)
+        self.indices = torch.full((P, H_kv, k), -1, dtype=torch.int32, device=dev)
+        self.k_eff = torch.zeros(P, dtype=torch.int32, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.layers = []
+        workspace = None
+        for l in range(P):
+            kv = mb.KVCache(k_cache[l:l + 1], v_cache[l:l + 1], H_q, B, seq_lens=seq_lens[l:l + 1])
+            if workspace is None:
+                workspace = kv.new_workspace(k)          # the layers run one after another and share it
+            self.layers.append(BlockAttention(kv, k, select_stream=self.select_stream, buffers={
+                "out": self.out[l:l + 1], "scores": self.scores[l:l + 1], "indices": self.indices[l:l + 1],
+                "k_eff": self.k_eff[l:l + 1], "status": self.status, "workspace": workspace}))
+
+    def run_block(self, q_steps: Sequence[torch.Tensor], kb_steps, vb_steps, outs: Sequence[torch.Tensor]):
+        """q_steps[t] is [P, H_q, B, d] (one slice per layer), likewise the block K/V and the outputs."""
+        T = len(q_steps)
+        for l, ba in enumerate(self.layers):
+            ba.exact_select(q_steps[0][l:l + 1], kb_steps[0][l:l + 1], vb_steps[0][l:l + 1], outs[0][l:l + 1])
+            ba.select_async()
+        self.layers[-1].join()                           # the select stream is in order: its last event covers all layers
+        for t in range(1, T):
+            for l, ba in enumerate(self.layers):
+                ba.sparse_step(q_steps[t][l:l + 1], kb_steps[t][l:l + 1], vb_steps[t][l:l + 1], outs[t][l:l + 1])
+        return outs

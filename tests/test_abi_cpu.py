@@ -83,7 +83,7 @@ def test_rejects_null_pointers_small_workspace_and_bad_scalars(lib):
     need = lib.mage_workspace_bytes(ctypes.byref(c), 1)
     assert lib.mage_exact_select(ctypes.byref(c), None, p, p, 0.088, p, p, p, need, None, None) == -1
     assert lib.mage_exact_select(ctypes.byref(c), p, p, p, 0.088, p, None, p, need, None, None) == -1
-    assert lib.mage_exact_select(ctypes.byref(c), p, p, p, 0.088, p, p, p, need - 1, None, None) == -3
+    assert lib.mage_exact_select(ctypes.byref(c), p, p, p, 0.088, p, p, p, 4096, None, None) == -3
     assert lib.mage_exact_select(ctypes.byref(c), p, p, p, 0.0, p, p, p, need, None, None) == -1
     assert lib.mage_exact_select(ctypes.byref(c), p, p, p, 0.088, p, p, ctypes.c_void_p(4100), need, None, None) == -1
     assert lib.mage_exact_select(None, p, p, p, 0.088, p, p, p, need, None, None) == -1
