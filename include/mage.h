@@ -53,6 +53,7 @@ typedef enum {
 #define MAGE_DEV_BAD_INDEX 1u   /* indices[] entry outside [0, N_p): row skipped    */
 #define MAGE_DEV_BAD_PAGE 2u    /* block_table entry outside [0, num_pages): skipped */
 #define MAGE_DEV_TIMEOUT 4u     /* an in-kernel bounded wait gave up                */
+#define MAGE_DEV_CACHE_FULL 8u  /* mage_append_block: no room left for the block: nothing appended for that problem */
 
 /* mage_kv_t.flags */
 #define MAGE_FLAG_SIMT_KERNELS 1  /* use the portable CUDA-core kernels for every stage (slow; for cross-checks) */
@@ -154,6 +155,21 @@ mage_status mage_sparse_block_attn(const mage_kv_t *kv, const void *q, const voi
                                    const int32_t *indices, const int32_t *k_eff, int32_t k, float sm_scale,
                                    void *out, void *workspace, size_t workspace_bytes, uint32_t *dev_status,
                                    void *stream);
+
+/*
+ * End of a block (Algorithm 1, last line: "C <- C || KV(x)"): append the finished block's keys and values to the
+ * prefix cache, so that the next block sees a prefix of N_p + B tokens.
+ *
+ *   k_blk, v_blk [P][H_kv][B][d] bf16   the block's final keys / values
+ *   seq_lens     [P] int32, device, in/out   N_p on entry, N_p + B on return (this argument, not kv->seq_lens, is
+ *                                            what is read and updated; it may be the same array)
+ * Rows go to logical positions N_p .. N_p+B-1: contiguous layout needs N_p + B <= N_max; paged layout needs the
+ * block table to map the pages those positions fall in already (the caller owns page allocation).  A problem that
+ * has no room, or whose page id is out of range, is left unchanged and MAGE_DEV_CACHE_FULL / MAGE_DEV_BAD_PAGE is
+ * set in *dev_status.  This is the one call that writes through kv->k_cache / kv->v_cache.
+ */
+mage_status mage_append_block(const mage_kv_t *kv, const void *k_blk, const void *v_blk, int32_t *seq_lens,
+                              uint32_t *dev_status, void *stream);
 
 /*
  * Step 1 of a block for callers that cannot hand over a workspace (the paper has no counterpart; this is a

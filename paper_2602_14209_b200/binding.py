@@ -18,7 +18,7 @@ _lib = None
 
 MAGE_OK = 0
 FLAG_SIMT_KERNELS = 1
-DEV_BAD_INDEX, DEV_BAD_PAGE, DEV_TIMEOUT = 1, 2, 4
+DEV_BAD_INDEX, DEV_BAD_PAGE, DEV_TIMEOUT, DEV_CACHE_FULL = 1, 2, 4, 8
 
 
 class MageError(RuntimeError):
@@ -38,7 +38,7 @@ class mage_kv_t(ctypes.Structure):
     ]
 
 
-EXPORTS = ("mage_workspace_bytes", "mage_exact_select", "mage_exact_select_events", "mage_exact_select_static", "mage_topk", "mage_sparse_block_attn",
+EXPORTS = ("mage_append_block", "mage_workspace_bytes", "mage_exact_select", "mage_exact_select_events", "mage_exact_select_static", "mage_topk", "mage_sparse_block_attn",
            "mage_status_string", "mage_launch_count")
 
 
@@ -63,6 +63,8 @@ def load():
     lib.mage_topk.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, ctypes.c_size_t, vp]
     lib.mage_sparse_block_attn.restype = ctypes.c_int
     lib.mage_sparse_block_attn.argtypes = [ctypes.POINTER(mage_kv_t), vp, vp, vp, vp, vp, i32, ctypes.c_float, vp, vp, ctypes.c_size_t, vp, vp]
+    lib.mage_append_block.restype = ctypes.c_int
+    lib.mage_append_block.argtypes = [ctypes.POINTER(mage_kv_t), vp, vp, vp, vp, vp]
     lib.mage_status_string.restype = ctypes.c_char_p
     lib.mage_status_string.argtypes = [ctypes.c_int]
     lib.mage_launch_count.restype = u64
@@ -189,3 +191,10 @@ def mage_sparse_block_attn(kv: KVCache, q, k_blk, v_blk, indices, k_eff, k: int,
                                        _ptr(dev_status), _stream(stream))
     if rc != MAGE_OK:
         raise MageError(rc, "mage_sparse_block_attn")
+
+
+def mage_append_block(kv: KVCache, k_blk, v_blk, seq_lens, dev_status=None, stream=None):
+    """End of a block: append the block's final K/V to the cache and add B to ``seq_lens`` (see mage.h)."""
+    rc = load().mage_append_block(ctypes.byref(kv.c), _ptr(k_blk), _ptr(v_blk), _ptr(seq_lens), _ptr(dev_status), _stream(stream))
+    if rc != MAGE_OK:
+        raise MageError(rc, "mage_append_block")

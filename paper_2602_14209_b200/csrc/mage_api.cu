@@ -269,6 +269,21 @@ mage_status mage_sparse_block_attn(const mage_kv_t *kv, const void *q, const voi
                        static_cast<float *>(workspace), ws_ok, dev_status, static_cast<cudaStream_t>(stream));
 }
 
+mage_status mage_append_block(const mage_kv_t *kv, const void *k_blk, const void *v_blk, int32_t *seq_lens, uint32_t *dev_status,
+                              void *stream) {
+    mage_status why = MAGE_OK;
+    if (!valid_kv(kv, &why)) return why;
+    if (!k_blk || !v_blk || !seq_lens || kv->N_max < 1) return MAGE_ERR_INVALID_ARG;
+    const KvView view = make_view(kv);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int warps = kv->P * kv->H_kv * kv->B;
+    append_rows_kernel<<<(warps + 3) / 4, 128, 0, st>>>(view, static_cast<const __nv_bfloat16 *>(k_blk), static_cast<const __nv_bfloat16 *>(v_blk),
+                                                       seq_lens, dev_status);
+    if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    bump_seq_lens_kernel<<<(kv->P + 127) / 128, 128, 0, st>>>(view, seq_lens);
+    return launch_check();
+}
+
 // Scratch for mage_exact_select_static.  In host code this name is only a handle for the runtime, not a device
 // address: the address is looked up once per device below and that pointer is what the kernels receive.
 static __device__ __align__(256) unsigned char g_static_scratch[MAGE_STATIC_SCRATCH_BYTES];

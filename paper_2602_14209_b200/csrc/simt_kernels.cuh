@@ -298,4 +298,53 @@ __global__ void __launch_bounds__(128) combine_kernel(KvView kv, Plan plan, floa
     *reinterpret_cast<uint2 *>(dst) = make_uint2(*reinterpret_cast<unsigned *>(&a), *reinterpret_cast<unsigned *>(&b));
 }
 
+// Cache append (Algorithm 1, "C <- C || KV(x)"): one warp per (problem, KV head, block token) copies the 256-byte
+// K row and V row to logical position N_p + token.  seq_lens is bumped by a second launch, after every row has
+// read the old length.
+__global__ void __launch_bounds__(128) append_rows_kernel(KvView kv, const __nv_bfloat16 *__restrict__ k_blk,
+                                                          const __nv_bfloat16 *__restrict__ v_blk, const int *__restrict__ seq_lens,
+                                                          unsigned *status) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    const int total = kv.P * kv.H_kv * kv.B;
+    if (warp >= total) return;
+    const int t = warp % kv.B, z = warp / kv.B, p = z / kv.H_kv, h = z % kv.H_kv;
+    const int n = seq_lens[p];
+    if (n < 0 || n + kv.B > kv.N_max) {
+        if (status && lane == 0) atomicOr(status, MAGE_DEV_CACHE_FULL);
+        return;
+    }
+    // every page the block touches must be mapped, or nothing of the block is written
+    if (kv.page_size) {
+        for (int j = n; j < n + kv.B; j += kv.page_size - (j % kv.page_size)) {
+            const int page = kv.block_table[(long long)p * kv.max_pages + j / kv.page_size];
+            if (page < 0 || page >= kv.num_pages) {
+                if (status && lane == 0) atomicOr(status, MAGE_DEV_BAD_PAGE);
+                return;
+            }
+        }
+    }
+    const long long off = cache_row_offset(kv, p, h, n + t, nullptr);
+    if (off < 0) return;
+    if (lane < 16) {
+        const uint4 kx = reinterpret_cast<const uint4 *>(k_blk + (long long)warp * kD)[lane];
+        const uint4 vx = reinterpret_cast<const uint4 *>(v_blk + (long long)warp * kD)[lane];
+        reinterpret_cast<uint4 *>(const_cast<__nv_bfloat16 *>(kv.k) + off)[lane] = kx;
+        reinterpret_cast<uint4 *>(const_cast<__nv_bfloat16 *>(kv.v) + off)[lane] = vx;
+    }
+}
+
+__global__ void bump_seq_lens_kernel(KvView kv, int *seq_lens) {
+    const int p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= kv.P) return;
+    const int n = seq_lens[p];
+    if (n < 0 || n + kv.B > kv.N_max) return;
+    if (kv.page_size) {
+        for (int j = n; j < n + kv.B; j += kv.page_size - (j % kv.page_size)) {
+            const int page = kv.block_table[(long long)p * kv.max_pages + j / kv.page_size];
+            if (page < 0 || page >= kv.num_pages) return;
+        }
+    }
+    seq_lens[p] = n + kv.B;
+}
+
 }  // namespace mage

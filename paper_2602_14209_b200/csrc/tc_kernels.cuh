@@ -156,6 +156,20 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
         const int per = (((rows + kScoreWgs - 1) / kScoreWgs) + 7) & ~7;
         const int col_lo = min(rows, wg * per), col_hi = min(rows, col_lo + per);
         const uint64_t c2 = pack2(scale_log2, scale_log2);
+        float prev_sum = 0.f;
+        // warpgroup 0: add the other warpgroups' partial sums of tile t to its own and store the score
+        auto finish = [&](int t, float own) -> bool {
+            const int b = t & 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(P_FULL + b), (t >> 1) & 1, abort_s, status))) return false;
+            float v = own;
+#pragma unroll
+            for (int g = 0; g < kScoreWgs - 1; ++g) v += part_s[(b * (kScoreWgs - 1) + g) * 128 + key];
+            mbar_arrive(bar(P_EMPTY + b));
+            v *= inv_m;
+            const int j = (tile0 + t) * kTile + key;
+            if (j < N) srow[j] = accumulate ? srow[j] + v : v;
+            return true;
+        };
         for (int i = 0; i < n_my; ++i) {
             const int buf = i & 1, ub = i >> 1;
             if (!__all_sync(0xffffffffu, mbar_wait(bar(T_FULL + buf), ub & 1, abort_s, status))) break;
@@ -206,16 +220,12 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                 part_s[(buf * (kScoreWgs - 1) + wg - 1) * 128 + key] = sum;
                 mbar_arrive(bar(P_FULL + buf));
             } else {
-                if (!__all_sync(0xffffffffu, mbar_wait(bar(P_FULL + buf), ub & 1, abort_s, status))) break;
-                float v = sum;
-#pragma unroll
-                for (int g = 0; g < kScoreWgs - 1; ++g) v += part_s[(buf * (kScoreWgs - 1) + g) * 128 + key];
-                mbar_arrive(bar(P_EMPTY + buf));
-                v *= inv_m;
-                const int j = (tile0 + i) * kTile + key;
-                if (j < N) srow[j] = accumulate ? srow[j] + v : v;
+                // warpgroup 0 completes tile i-1 here, one tile late, so that it never waits for the others' partial sums
+                if (i > 0 && !finish(i - 1, prev_sum)) break;
+                prev_sum = sum;
             }
         }
+        if (wg == 0 && n_my > 0) finish(n_my - 1, prev_sum);
     }
     tc_fence_before_sync();
     __syncthreads();

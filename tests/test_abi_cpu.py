@@ -93,6 +93,9 @@ def test_rejects_null_pointers_small_workspace_and_bad_scalars(lib):
     assert lib.mage_topk(p, None, 0, 2, 2048, 8, p, p, None, 0, None) == -1
     assert lib.mage_topk(p, None, 1, 2, 2048, 8, None, p, None, 0, None) == -1
     assert lib.mage_topk(None, None, 1, 2, 2048, 8, p, p, None, 0, None) == -1
+    assert lib.mage_append_block(ctypes.byref(c), p, p, None, None, None) == -1
+    assert lib.mage_append_block(ctypes.byref(c), None, p, p, None, None) == -1
+    assert lib.mage_append_block(None, p, p, p, None, None) == -1
 
 
 def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
