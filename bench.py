@@ -382,6 +382,43 @@ def main():
                 stages["layerwise_cuda_graph_error"] = str(e)[:200]
             stages["layerwise_dev_status"] = int(lw.status.item())
 
+        # Serving batch (ragged, paged): one scheduler tick with the sequences staggered over the T steps of a block.
+        # Two sequences are at Step 1 (exact_select on the main stream, their top-k on the select stream), the other
+        # fourteen take a reuse step on the main stream meanwhile.  Reported with the top-k overlapped and, for
+        # comparison, with everything serialised on the main stream.
+        if w.page_size and w.P >= 4:
+            n1 = max(1, w.P // T)
+            idx1 = torch.arange(0, n1, device=dev)
+            idx2 = torch.arange(n1, w.P, device=dev)
+            sub = lambda idx: mb.KVCache(k_pool, v_pool, w.H_q, w.B, seq_lens=batch["seq_lens"][idx].contiguous(),
+                                         block_table=table[idx].contiguous(), N_max=batch["N_max"], flags=flags)
+            ba1, ba2 = BlockAttention(sub(idx1), w.k), BlockAttention(sub(idx2), w.k)
+            q1, kb1, vb1 = q_d[0][:n1].contiguous(), kb_d[0][:n1].contiguous(), vb_d[0][:n1].contiguous()
+            q2, kb2, vb2 = q_d[1][n1:].contiguous(), kb_d[1][n1:].contiguous(), vb_d[1][n1:].contiguous()
+            ba2.run_block([q2, q2], [kb2, kb2], [vb2, vb2])          # gives group 2 a valid index set
+            torch.cuda.synchronize()
+
+            def tick(overlap):
+                ba1.exact_select(q1, kb1, vb1)
+                if overlap:
+                    ba1.select_async()
+                else:
+                    mb.mage_topk(ba1.scores, ba1.kv.seq_lens, ba1.kv.P, ba1.kv.H_kv, ba1.kv.N_max, w.k, ba1.indices, ba1.k_eff)
+                ba2.sparse_step(q2, kb2, vb2)
+                if overlap:
+                    ba1.join()
+
+            for mode in (True, False):
+                for _ in range(3):
+                    tick(mode)
+                torch.cuda.synchronize()
+                a.record()
+                for _ in range(20):
+                    tick(mode)
+                b.record(); torch.cuda.synchronize()
+                stages["serving_tick_ms_topk_on_select_stream" if mode else "serving_tick_ms_serialised"] = a.elapsed_time(b) / 20
+            stages["serving_tick_groups"] = f"{n1} sequences at Step 1 + {w.P - n1} at a reuse step"
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
