@@ -85,9 +85,9 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
         for (int s = 0; s < kScoreStages; ++s) { mbar_init(bar(FULL + s), 1); mbar_init(bar(EMPTY + s), 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(T_FULL + b), 1);
-            mbar_init(bar(T_EMPTY + b), kScoreWgs * 128);
-            mbar_init(bar(P_FULL + b), (kScoreWgs - 1) * 128);
-            mbar_init(bar(P_EMPTY + b), 128);
+            mbar_init(bar(T_EMPTY + b), kScoreWgs * 4);            // one arrival per warp
+            mbar_init(bar(P_FULL + b), (kScoreWgs - 1) * 4);
+            mbar_init(bar(P_EMPTY + b), 4);
         }
         fence_mbar_init();
     }
@@ -164,7 +164,7 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
             float v = own;
 #pragma unroll
             for (int g = 0; g < kScoreWgs - 1; ++g) v += part_s[(b * (kScoreWgs - 1) + g) * 128 + key];
-            mbar_arrive(bar(P_EMPTY + b));
+            mbar_arrive_warp(bar(P_EMPTY + b));
             v *= inv_m;
             const int j = (tile0 + t) * kTile + key;
             if (j < N) srow[j] = accumulate ? srow[j] + v : v;
@@ -211,14 +211,14 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                 }
             }
             tc_fence_before_sync();
-            mbar_arrive(bar(T_EMPTY + buf));
+            mbar_arrive_warp(bar(T_EMPTY + buf));
             float a0, a1, b0, b1;
             unpack2(acc_a, a0, a1); unpack2(acc_b, b0, b1);
             const float sum = ((a0 + a1) + (b0 + b1)) + tail;
             if (wg > 0) {
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(P_EMPTY + buf), (ub & 1) ^ 1, abort_s, status))) break;
                 part_s[(buf * (kScoreWgs - 1) + wg - 1) * 128 + key] = sum;
-                mbar_arrive(bar(P_FULL + buf));
+                mbar_arrive_warp(bar(P_FULL + buf));
             } else {
                 // warpgroup 0 completes tile i-1 here, one tile late, so that it never waits for the others' partial sums
                 if (i > 0 && !finish(i - 1, prev_sum)) break;
@@ -318,11 +318,11 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
     if (tid == 0) {
         *abort_s = 0;
         mbar_init(bar(Q_FULL), 1);
-        for (int s = 0; s < kAttnSlots; ++s) { mbar_init(bar(FULL + s), SPARSE ? 128 : 1); mbar_init(bar(EMPTY + s), 1); }
+        for (int s = 0; s < kAttnSlots; ++s) { mbar_init(bar(FULL + s), SPARSE ? 4 : 1); mbar_init(bar(EMPTY + s), 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(S_FULL + b), 1);
-            mbar_init(bar(P_HALF + b), 128);
-            mbar_init(bar(P_FULL + b), 128);
+            mbar_init(bar(P_HALF + b), 4);                  // one arrival per warp
+            mbar_init(bar(P_FULL + b), 4);
             mbar_init(bar(PVH_DONE + b), 1);
         }
         mbar_init(bar(O_DONE), 1);
@@ -411,18 +411,18 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 if (L >= 2) {
                     cp_async_wait<2>();
                     fence_proxy_async();
-                    mbar_arrive(bar(FULL + slot_of(L - 2)));
+                    mbar_arrive_warp(bar(FULL + slot_of(L - 2)));
                 }
             }
             if (ok) {
                 if (issued >= 2) {
                     cp_async_wait<1>();
                     fence_proxy_async();
-                    mbar_arrive(bar(FULL + slot_of(issued - 2)));
+                    mbar_arrive_warp(bar(FULL + slot_of(issued - 2)));
                 }
                 cp_async_wait<0>();
                 fence_proxy_async();
-                mbar_arrive(bar(FULL + slot_of(issued - 1)));
+                mbar_arrive_warp(bar(FULL + slot_of(issued - 1)));
             } else {
                 cp_async_wait<0>();
             }
@@ -579,7 +579,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                         tmem_ld32(tS + 96, rb);
                         tmem_wait_st();
                         tc_fence_before_sync();
-                        mbar_arrive(bar(P_HALF + mt));         // the PV MMA may start on keys 0-63
+                        mbar_arrive_warp(bar(P_HALF + mt));    // the PV MMA may start on keys 0-63
                         half_done = true;
                         // second half (keys 64-127): its P lands on S columns 32-63, already consumed; its own S
                         // columns 64-127 are never overwritten
@@ -708,8 +708,8 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     fence_proxy_async();
                 }
                 tc_fence_before_sync();
-                if (!half_done) mbar_arrive(bar(P_HALF + mt));
-                mbar_arrive(bar(P_FULL + mt));
+                if (!half_done) mbar_arrive_warp(bar(P_HALF + mt));
+                mbar_arrive_warp(bar(P_FULL + mt));
             }
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(O_DONE), 0, abort_s, status));
             if (ok) {
