@@ -39,18 +39,22 @@ __device__ __forceinline__ void cache_box_coords(const KvView &kv, int p, int h,
 // Block-score kernel (Eq. 4): score[j] = 1/M * sum_r exp2(scale_log2 * <q_r, k_j> - lse2_r).
 // Orientation: keys are the MMA M dimension (TMEM lanes), query rows the N dimension (TMEM columns), so each
 // thread owns one key and its sum over rows needs no cross-thread reduction.  One CTA walks `tiles_per_cta`
-// consecutive 128-key tiles of one KV head; S^T tiles are double-buffered in TMEM.
+// consecutive 128-key tiles of one KV head.
 // The kernel is bound by the special-function unit (128*M exponentials per tile at 16 per clock per SM, against
-// 4*M clocks of MMA), so the job of the layout is to keep that unit fed: kScoreWgs warpgroups (four warps per
-// scheduler) all work on every tile, each on a slice of the columns (query rows); warpgroups 1.. hand their 128
-// partial sums to warpgroup 0 through shared memory, which adds them in a fixed order.
+// 4*M clocks of MMA), so the layout's job is to keep that unit busy through the hand-offs.  A unit of work is
+// (key tile, half of the query rows): S^T of a unit is 128 lanes x <=128 columns, TMEM holds four of them, and each
+// of the four warpgroups owns one buffer: warpgroup w takes the units u = w (mod 4), i.e. tiles of parity w/2 and
+// row half w%2.  While one warpgroup waits for the MMA to refill its buffer the other three are in their
+// exponentials, so the hand-off latency is hidden without any warpgroup-to-warpgroup barrier.  The row-half-1
+// warpgroup of a tile hands its 128 partial sums to the row-half-0 warpgroup through shared memory, which adds them
+// (fixed order) one unit late and stores the score.
 // ------------------------------------------------------------------------------------------------------------
 constexpr int kScoreStages = 4;
 constexpr int kScoreWgs = 4;
 constexpr int kScoreThreads = kScoreWgs * 128 + 64;
 constexpr int kScoreProducerWarp = kScoreWgs * 4, kScoreMmaWarp = kScoreWgs * 4 + 1;
 constexpr int kScoreQBytes = 2 * 256 * 128;           // up to 256 query rows, two d-halves
-constexpr size_t kScoreSmemBytes = 1024 + kScoreQBytes + kScoreStages * kTileBytes + (256 + 2 * (kScoreWgs - 1) * 128) * sizeof(float) + 256;
+constexpr size_t kScoreSmemBytes = 1024 + kScoreQBytes + kScoreStages * kTileBytes + (256 + 2 * 128) * sizeof(float) + 256;
 
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, KvView kv, Plan plan,
@@ -68,27 +72,26 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *q_s = base, *k_s = base + kScoreQBytes;
     float *neg_lse_s = reinterpret_cast<float *>(k_s + kScoreStages * kTileBytes);
-    float *part_s = neg_lse_s + 256;                   // [2][kScoreWgs-1][128] partial sums of warpgroups 1..
-    uint64_t *bars = reinterpret_cast<uint64_t *>(part_s + 2 * (kScoreWgs - 1) * 128);
-    enum { Q_FULL = 0, FULL = 1, EMPTY = FULL + kScoreStages, T_FULL = EMPTY + kScoreStages, T_EMPTY = T_FULL + 2,
-           P_FULL = T_EMPTY + 2, P_EMPTY = P_FULL + 2, N_BARS = P_EMPTY + 2 };
+    float *part_s = neg_lse_s + 256;                   // [2 tile parities][128] partial sums of the row-half-1 warpgroups
+    uint64_t *bars = reinterpret_cast<uint64_t *>(part_s + 2 * 128);
+    enum { Q_FULL = 0, FULL = 1, EMPTY = FULL + kScoreStages, T_FULL = EMPTY + kScoreStages, T_EMPTY = T_FULL + 4,
+           P_FULL = T_EMPTY + 4, P_EMPTY = P_FULL + 2, N_BARS = P_EMPTY + 2 };
     uint32_t *tmem_ptr_s = reinterpret_cast<uint32_t *>(bars + N_BARS);
     volatile int *abort_s = reinterpret_cast<volatile int *>(tmem_ptr_s + 1);
     auto bar = [&](int i) { return smem_u32(bars + i); };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int rows64 = (rows + 63) & ~63, n_mma = (rows + 15) & ~15;
+    const int rows64 = (rows + 63) & ~63;
+    // the two row halves: [0, rows_lo) and [rows_lo, rows); rows_lo is a multiple of 8 rows (one swizzle atom)
+    const int rows_lo = min(rows, (((rows + 1) >> 1) + 7) & ~7), rows_hi = rows - rows_lo;
+    const int n_units = rows_hi > 0 ? 2 : 1;           // units per tile
 
     if (tid == 0) {
         *abort_s = 0;
         mbar_init(bar(Q_FULL), 1);
         for (int s = 0; s < kScoreStages; ++s) { mbar_init(bar(FULL + s), 1); mbar_init(bar(EMPTY + s), 1); }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(bar(T_FULL + b), 1);
-            mbar_init(bar(T_EMPTY + b), kScoreWgs * 4);            // one arrival per warp
-            mbar_init(bar(P_FULL + b), (kScoreWgs - 1) * 4);
-            mbar_init(bar(P_EMPTY + b), 4);
-        }
+        for (int b = 0; b < 4; ++b) { mbar_init(bar(T_FULL + b), 1); mbar_init(bar(T_EMPTY + b), 4); }   // one arrival per warp
+        for (int b = 0; b < 2; ++b) { mbar_init(bar(P_FULL + b), 4); mbar_init(bar(P_EMPTY + b), 4); }
         fence_mbar_init();
     }
     if (warp == kScoreMmaWarp) { tmem_alloc(smem_u32(tmem_ptr_s), 512); tmem_relinquish(); }
@@ -130,102 +133,109 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
         }
     } else if (warp == kScoreMmaWarp) {
         if (lane == 0) {
-            const uint32_t idesc = idesc_bf16_f32(n_mma, false, false);
+            const uint32_t idesc_lo = idesc_bf16_f32((rows_lo + 15) & ~15, false, false);
+            const uint32_t idesc_hi = idesc_bf16_f32(max(16, (rows_hi + 15) & ~15), false, false);
             bool ok = mbar_wait(bar(Q_FULL), 0, abort_s, status);
             for (int i = 0; ok && i < n_my; ++i) {
-                const int slot = i % kScoreStages, u = i / kScoreStages, buf = i & 1, ub = i >> 1;
-                if (!mbar_wait(bar(T_EMPTY + buf), (ub & 1) ^ 1, abort_s, status)) break;
-                if (!mbar_wait(bar(FULL + slot), u & 1, abort_s, status)) break;
-                tc_fence_after_sync();
+                const int slot = i % kScoreStages, su = i / kScoreStages;
+                if (!mbar_wait(bar(FULL + slot), su & 1, abort_s, status)) break;
                 const uint32_t k_addr = smem_u32(k_s + slot * kTileBytes), q_addr = smem_u32(q_s);
+                for (int rh = 0; rh < n_units && ok; ++rh) {
+                    const int buf = (i & 1) * 2 + rh, use = i >> 1;          // buffer = warpgroup that consumes it
+                    if (!mbar_wait(bar(T_EMPTY + buf), (use & 1) ^ 1, abort_s, status)) { ok = false; break; }
+                    tc_fence_after_sync();
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t a = smem_desc_sw128(k_addr + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
-                    const uint64_t b = smem_desc_sw128(q_addr + (ks >> 2) * (kScoreQBytes / 2) + (ks & 3) * 32, 16, 1024);
-                    umma_ss(tmem_base + buf * 256, a, b, idesc, ks > 0);
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+                        const uint64_t a = smem_desc_sw128(k_addr + off, 16, 1024);
+                        const uint64_t b = smem_desc_sw128(q_addr + (ks >> 2) * (kScoreQBytes / 2) + (ks & 3) * 32 + rh * rows_lo * 128, 16, 1024);
+                        umma_ss(tmem_base + buf * 128, a, b, rh ? idesc_hi : idesc_lo, ks > 0);
+                    }
+                    umma_commit(bar(T_FULL + buf));
                 }
                 umma_commit(bar(EMPTY + slot));
-                umma_commit(bar(T_FULL + buf));
             }
         }
     } else {
         const int wg = warp >> 2, w4 = warp & 3, key = w4 * 32 + lane;
+        const int par = wg >> 1, rh = wg & 1;               // tile parity and row half of this warpgroup
         const float inv_m = 1.f / (float)kv.M;
         float *srow = scores + (size_t)z * kv.N_max;
-        // column slice of this warpgroup, in units of 8 columns
-        const int per = (((rows + kScoreWgs - 1) / kScoreWgs) + 7) & ~7;
-        const int col_lo = min(rows, wg * per), col_hi = min(rows, col_lo + per);
+        const int col_lo = rh ? rows_lo : 0, n_cols = rh ? rows_hi : rows_lo;      // my columns: neg_lse index = col_lo + c
         const uint64_t c2 = pack2(scale_log2, scale_log2);
+        const uint32_t taddr = tmem_base + wg * 128 + ((uint32_t)(w4 * 32) << 16);
         float prev_sum = 0.f;
-        // warpgroup 0: add the other warpgroups' partial sums of tile t to its own and store the score
+        int prev_tile = -1;
+        // row half 0: add the other half's partial sum of tile t to its own and store the score
         auto finish = [&](int t, float own) -> bool {
-            const int b = t & 1;
-            if (!__all_sync(0xffffffffu, mbar_wait(bar(P_FULL + b), (t >> 1) & 1, abort_s, status))) return false;
             float v = own;
-#pragma unroll
-            for (int g = 0; g < kScoreWgs - 1; ++g) v += part_s[(b * (kScoreWgs - 1) + g) * 128 + key];
-            mbar_arrive_warp(bar(P_EMPTY + b));
+            if (n_units == 2) {
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(P_FULL + par), (t >> 1) & 1, abort_s, status))) return false;
+                v += part_s[par * 128 + key];
+                mbar_arrive_warp(bar(P_EMPTY + par));
+            }
             v *= inv_m;
             const int j = (tile0 + t) * kTile + key;
             if (j < N) srow[j] = accumulate ? srow[j] + v : v;
             return true;
         };
-        for (int i = 0; i < n_my; ++i) {
-            const int buf = i & 1, ub = i >> 1;
-            if (!__all_sync(0xffffffffu, mbar_wait(bar(T_FULL + buf), ub & 1, abort_s, status))) break;
-            tc_fence_after_sync();
-            float tail = 0.f;
-            uint64_t acc_a = pack2(0.f, 0.f), acc_b = acc_a;
-            const uint32_t taddr = tmem_base + buf * 256 + ((uint32_t)(w4 * 32) << 16);
-            // one unit = 8 columns = 4 pairs; the TMEM load of the next unit is in flight while this one is processed
-            auto unit = [&](const uint32_t (&r)[8], int c0) {
-                if (c0 + 8 <= col_hi) {
-                    const float4 *nl4 = reinterpret_cast<const float4 *>(neg_lse_s + c0);
-                    const float4 n0 = nl4[0], n1 = nl4[1];
-                    uint64_t x[4];
-                    x[0] = fma2(pack2(__uint_as_float(r[0]), __uint_as_float(r[1])), c2, pack2(n0.x, n0.y));
-                    x[1] = fma2(pack2(__uint_as_float(r[2]), __uint_as_float(r[3])), c2, pack2(n0.z, n0.w));
-                    x[2] = fma2(pack2(__uint_as_float(r[4]), __uint_as_float(r[5])), c2, pack2(n1.x, n1.y));
-                    x[3] = fma2(pack2(__uint_as_float(r[6]), __uint_as_float(r[7])), c2, pack2(n1.z, n1.w));
-                    ex2_mufu2_n(x);
-                    acc_a = add2(acc_a, x[0]); acc_b = add2(acc_b, x[1]);
-                    acc_a = add2(acc_a, x[2]); acc_b = add2(acc_b, x[3]);
-                } else {
+        bool ok = true;
+        if (n_cols > 0) {
+            for (int i = par; i < n_my; i += 2) {
+                const int use = i >> 1;
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(T_FULL + wg), use & 1, abort_s, status))) { ok = false; break; }
+                tc_fence_after_sync();
+                float tail = 0.f;
+                uint64_t acc_a = pack2(0.f, 0.f), acc_b = acc_a;
+                // one step = 8 columns = 4 pairs; the TMEM load of the next step is in flight while this one is processed
+                auto step = [&](const uint32_t (&r)[8], int c0) {
+                    if (c0 + 8 <= n_cols) {
+                        const float4 *nl4 = reinterpret_cast<const float4 *>(neg_lse_s + col_lo + c0);
+                        const float4 n0 = nl4[0], n1 = nl4[1];
+                        uint64_t x[4];
+                        x[0] = fma2(pack2(__uint_as_float(r[0]), __uint_as_float(r[1])), c2, pack2(n0.x, n0.y));
+                        x[1] = fma2(pack2(__uint_as_float(r[2]), __uint_as_float(r[3])), c2, pack2(n0.z, n0.w));
+                        x[2] = fma2(pack2(__uint_as_float(r[4]), __uint_as_float(r[5])), c2, pack2(n1.x, n1.y));
+                        x[3] = fma2(pack2(__uint_as_float(r[6]), __uint_as_float(r[7])), c2, pack2(n1.z, n1.w));
+                        ex2_mufu2_n(x);
+                        acc_a = add2(acc_a, x[0]); acc_b = add2(acc_b, x[1]);
+                        acc_a = add2(acc_a, x[2]); acc_b = add2(acc_b, x[3]);
+                    } else {
 #pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        if (c0 + e < col_hi) tail += ex2(fmaf(__uint_as_float(r[e]), scale_log2, neg_lse_s[c0 + e]));
-                }
-            };
-            if (col_lo < col_hi) {
+                        for (int e = 0; e < 8; ++e)
+                            if (c0 + e < n_cols) tail += ex2(fmaf(__uint_as_float(r[e]), scale_log2, neg_lse_s[col_lo + c0 + e]));
+                    }
+                };
                 uint32_t ra[8], rb[8];
-                tmem_ld8(taddr + col_lo, ra);
-                for (int c0 = col_lo; c0 < col_hi; c0 += 16) {
+                tmem_ld8(taddr, ra);
+                for (int c0 = 0; c0 < n_cols; c0 += 16) {
                     tmem_wait_ld(ra);
-                    if (c0 + 8 < col_hi) tmem_ld8(taddr + c0 + 8, rb);
-                    unit(ra, c0);
-                    if (c0 + 8 < col_hi) {
+                    if (c0 + 8 < n_cols) tmem_ld8(taddr + c0 + 8, rb);
+                    step(ra, c0);
+                    if (c0 + 8 < n_cols) {
                         tmem_wait_ld(rb);
-                        if (c0 + 16 < col_hi) tmem_ld8(taddr + c0 + 16, ra);
-                        unit(rb, c0 + 8);
+                        if (c0 + 16 < n_cols) tmem_ld8(taddr + c0 + 16, ra);
+                        step(rb, c0 + 8);
                     }
                 }
+                tc_fence_before_sync();
+                mbar_arrive_warp(bar(T_EMPTY + wg));
+                float a0, a1, b0, b1;
+                unpack2(acc_a, a0, a1); unpack2(acc_b, b0, b1);
+                const float sum = ((a0 + a1) + (b0 + b1)) + tail;
+                if (rh == 1) {
+                    if (!__all_sync(0xffffffffu, mbar_wait(bar(P_EMPTY + par), (use & 1) ^ 1, abort_s, status))) { ok = false; break; }
+                    part_s[par * 128 + key] = sum;
+                    mbar_arrive_warp(bar(P_FULL + par));
+                } else {
+                    // finish the previous tile of this parity now, one unit late, so this warpgroup never waits for its partner
+                    if (prev_tile >= 0 && !finish(prev_tile, prev_sum)) { ok = false; break; }
+                    prev_sum = sum;
+                    prev_tile = i;
+                }
             }
-            tc_fence_before_sync();
-            mbar_arrive_warp(bar(T_EMPTY + buf));
-            float a0, a1, b0, b1;
-            unpack2(acc_a, a0, a1); unpack2(acc_b, b0, b1);
-            const float sum = ((a0 + a1) + (b0 + b1)) + tail;
-            if (wg > 0) {
-                if (!__all_sync(0xffffffffu, mbar_wait(bar(P_EMPTY + buf), (ub & 1) ^ 1, abort_s, status))) break;
-                part_s[(buf * (kScoreWgs - 1) + wg - 1) * 128 + key] = sum;
-                mbar_arrive_warp(bar(P_FULL + buf));
-            } else {
-                // warpgroup 0 completes tile i-1 here, one tile late, so that it never waits for the others' partial sums
-                if (i > 0 && !finish(i - 1, prev_sum)) break;
-                prev_sum = sum;
-            }
+            if (ok && rh == 0 && prev_tile >= 0) finish(prev_tile, prev_sum);
         }
-        if (wg == 0 && n_my > 0) finish(n_my - 1, prev_sum);
     }
     tc_fence_before_sync();
     __syncthreads();
