@@ -1,8 +1,9 @@
 // Tensor-core (tcgen05 + TMEM + TMA) kernels of the path for sm_100a.
 //
-// Warp roles in every kernel here: warps 0-3 and 4-7 are two "softmax" warpgroups (warp w owns TMEM lanes
-// 32*(w%4)..+31), one producer warp issues TMA tile loads, one warp issues tcgen05.mma from a single lane and
-// owns the TMEM allocation.  All hand-offs go through mbarriers with bounded waits (sm100_ptx.cuh).
+// Warp roles in every kernel here: the first warps form "softmax" warpgroups of four warps (warp w owns TMEM lanes
+// 32*(w%4)..+31: two warpgroups in the attention kernel, four in the score kernel), then come the producer warp(s)
+// that issue TMA tile loads or gather rows with cp.async, and one warp that issues tcgen05.mma from a single lane
+// and owns the TMEM allocation.  All hand-offs go through mbarriers with bounded waits (sm100_ptx.cuh).
 #pragma once
 #include "common.cuh"
 #include "sm100_ptx.cuh"

@@ -156,3 +156,40 @@ def test_logit_jumps_beyond_the_lazy_rescale_range(oracle_mod, flags):
     H.check_problem(oracle_mod, batch, res, w, 0, check_topk=False, o_max_abs=2e-2)
     # the dominant key takes (almost) all of the probability mass of every row
     assert abs(res["scores"][0, 0, 700] - 1.0) < 1e-5 and res["scores"][0, 0, :700].max() < 1e-30
+
+
+def test_layer_by_layer_runner_matches_batched_runner(oracle_mod):
+    """pipeline.LayerwiseBlock (one launch per layer, P = 1 views of the same memory) against the batched call."""
+    from paper_2602_14209_b200.pipeline import LayerwiseBlock
+    w = W.Workload("layers", H_q=8, H_kv=2, N=3000, B=32, k=128, T=3, P=4, n_heavy=16, seed=17)
+    batch = W.make_batch(w, device="cuda")
+    res = H.run_gpu_block(batch, w)
+    lw = LayerwiseBlock(batch["kc"], batch["vc"], w.H_q, w.B, w.k, batch["seq_lens"])
+    outs = [torch.full_like(lw.out, float("nan")) for _ in range(w.T)]
+    lw.run_block([batch["q"][t] for t in range(w.T)], [batch["kb"][t] for t in range(w.T)], [batch["vb"][t] for t in range(w.T)], outs)
+    torch.cuda.synchronize()
+    assert int(lw.status.item()) == 0
+    res_lw = {"outs": [o.float().cpu().numpy() for o in outs], "scores": lw.scores.cpu().numpy(), "indices": lw.indices.cpu().numpy(),
+              "k_eff": lw.k_eff.cpu().numpy(), "status": 0, "k": w.k}
+    res_lw["scores"][:, :, w.N:] = -1.0
+    for p in range(w.P):
+        H.check_problem(oracle_mod, batch, res_lw, w, p)
+        assert np.abs(res_lw["outs"][0][p] - res["outs"][0][p]).max() < 1e-2
+
+
+def test_sparse_step_without_workspace_and_events_variant(oracle_mod):
+    """mage_sparse_block_attn accepts a null workspace (no split across CTAs); mage_exact_select_events records its events."""
+    w = W.CONFIGS["cfg1_small"]
+    batch = W.make_batch(w, device="cuda")
+    res = H.run_gpu_block(batch, w)
+    ba = res["ba"]
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    ba.exact_select(batch["q"][0], batch["kb"][0], batch["vb"][0], events=ev)
+    out_a = ba.sparse_step(batch["q"][1], batch["kb"][1], batch["vb"][1]).clone()
+    out_b = torch.empty_like(out_a)
+    mb.mage_sparse_block_attn(ba.kv, batch["q"][1], batch["kb"][1], batch["vb"][1], ba.indices, ba.k_eff, ba.k, ba.sm_scale, out_b,
+                              None, ba.status)
+    torch.cuda.synchronize()
+    assert ev[0].elapsed_time(ev[3]) > 0 and ev[0].elapsed_time(ev[1]) > 0
+    assert (out_a.float() - out_b.float()).abs().max() < 5e-3
+    assert np.abs(out_b.float().cpu().numpy() - res["outs"][1]).max() < 5e-3
