@@ -518,6 +518,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             const uint32_t lane_off = (uint32_t)(w4 * 32) << 16;
             const uint32_t tS = tmem_base + mt * 128 + lane_off, tO = tmem_base + 256 + mt * 128 + lane_off;
             const int row = w4 * 32 + lane, grow = rg * 256 + mt * kTile + row;
+            const bool warp_has_rows = rg * 256 + mt * kTile + w4 * 32 < kv.M;
             float m_used = -INFINITY, l = 0.f;
             float pend_m = 0.f;          // reference the row wants to move to at the start of its next tile
             bool pending = false;
@@ -541,8 +542,9 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     }
                     tmem_wait_st();
                 };
+                // a warp whose 32 rows all lie beyond M (row padding of the last M-tile) only takes part in the hand-offs
                 bool fast = i > 0 && valid == kTile, half_done = false;
-                if (fast) {
+                if (warp_has_rows && fast) {
                     // ---- common case: one sweep over S with the reference maximum carried over from earlier tiles.
                     // exp2(x - m_used) stays representable as long as x - m_used < 100, so the true maximum is only
                     // tracked (to move the reference lazily, at the next tile) and checked against that limit.
@@ -646,7 +648,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                         tmem_st16(tS + 48, pb);
                     }
                 }
-                if (!fast) {
+                if (warp_has_rows && !fast) {
                     // ---- careful path (first tile, ragged last tile, or a jump of the maximum by more than 2^100):
                     // find the tile's maximum first, move the reference if it grew, then exponentiate.
                     float mx = -INFINITY;
