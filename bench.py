@@ -166,6 +166,8 @@ def main():
     ap.add_argument("--simt", action="store_true", help="force the portable CUDA-core kernels")
     ap.add_argument("--P", type=int, default=None, help="override the number of problems (layers/sequences) of the workload")
     ap.add_argument("--N", type=int, default=None, help="override the prefix length of the workload")
+    ap.add_argument("--ragged-min", type=int, default=None,
+                    help="override the lower bound of the per-sequence prefix lengths (0 = every sequence has N tokens)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-stage-breakdown", action="store_true")
     args = ap.parse_args()
@@ -176,6 +178,9 @@ def main():
     if args.P is not None or args.N is not None:
         import dataclasses as _dc
         w = _dc.replace(w, P=args.P or w.P, N=args.N or w.N, name=f"{w.name}[P={args.P or w.P},N={args.N or w.N}]")
+    if args.ragged_min is not None:
+        import dataclasses as _dc
+        w = _dc.replace(w, ragged_min=args.ragged_min, name=f"{w.name}[ragged_min={args.ragged_min}]")
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -311,13 +311,17 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
     }
     const int n_tiles = (n_keys + kTile - 1) / kTile;
     const int rows_here = min(256, kv.M - rg * 256), n_mt = rows_here > 128 ? 2 : 1;
+    // With a single M-tile the second softmax warpgroup and the second S/O regions would idle.  They take the
+    // odd key tiles instead ("tile-parity mode"): two independent online-softmax pipelines over the same 128 rows,
+    // each with its own reference, sum and O accumulator, merged by warpgroup 0 at the end.
+    const bool tp = n_mt == 1;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *q_s = base, *kv_s = base + kAttnQBytes;
     uint64_t *bars = reinterpret_cast<uint64_t *>(kv_s + kAttnSlots * kTileBytes);
     enum { Q_FULL = 0, FULL = 1, EMPTY = FULL + kAttnSlots, S_FULL = EMPTY + kAttnSlots, P_HALF = S_FULL + 2, P_FULL = P_HALF + 2,
-           PVH_DONE = P_FULL + 2, O_DONE = PVH_DONE + 2, N_BARS = O_DONE + 1 };
+           PVH_DONE = P_FULL + 2, O_DONE = PVH_DONE + 2, PUB = O_DONE + 1, N_BARS = PUB + 1 };
     uint32_t *tmem_ptr_s = reinterpret_cast<uint32_t *>(bars + N_BARS);
     volatile int *abort_s = reinterpret_cast<volatile int *>(tmem_ptr_s + 1);
     int *row_tab = reinterpret_cast<int *>(tmem_ptr_s + 4);     // SPARSE: cache offset / 8 of each selected row, -1 = skip
@@ -337,6 +341,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             mbar_init(bar(PVH_DONE + b), 1);
         }
         mbar_init(bar(O_DONE), 1);
+        mbar_init(bar(PUB), 4);
         fence_mbar_init();
     }
     if (warp == kMmaWarp) { tmem_alloc(smem_u32(tmem_ptr_s), 512); tmem_relinquish(); }
@@ -452,13 +457,15 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             const uint32_t idesc_qk = idesc_bf16_f32(kTile, false, false);   // S[128 rows][128 keys]
             const uint32_t idesc_pv = idesc_bf16_f32(kD, false, true);       // O[128 rows][128 d], V is MN-major
             const uint32_t q_addr = smem_u32(q_s);
-            auto qk = [&](int i, int mt) {
+            // reg = which S/O region (and softmax warpgroup); the Q tile is reg with two M-tiles, tile 0 in tile-parity mode
+            auto qk = [&](int i, int reg) {
                 const uint32_t k_addr = smem_u32(kv_s + slot_of(2 * i) * kTileBytes);
+                const uint32_t qt = tp ? 0 : reg;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t a = smem_desc_sw128(q_addr + mt * kTileBytes + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
+                    const uint64_t a = smem_desc_sw128(q_addr + qt * kTileBytes + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
                     const uint64_t b = smem_desc_sw128(k_addr + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
-                    umma_ss(tmem_base + mt * 128, a, b, idesc_qk, ks > 0);
+                    umma_ss(tmem_base + reg * 128, a, b, idesc_qk, ks > 0);
                 }
             };
             auto pv = [&](int i, int mt, int half) {  // half 0: keys 0-63 of the tile, half 1: keys 64-127
@@ -466,10 +473,40 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
 #pragma unroll
                 for (int ks = half * 4; ks < half * 4 + 4; ++ks) {      // 16 keys per step: 16 rows of 128 bytes in each d-half
                     const uint64_t b = smem_desc_sw128(v_addr + ks * 2048, kHalfBytes, 1024);
-                    umma_ts(tmem_base + 256 + mt * 128, tmem_base + mt * 128 + ks * 8, b, idesc_pv, (i > 0 || ks > 0) ? 1u : 0u);
+                    umma_ts(tmem_base + 256 + mt * 128, tmem_base + mt * 128 + ks * 8, b, idesc_pv, (i > (tp ? 1 : 0) || ks > 0) ? 1u : 0u);
                 }
             };
             bool ok = mbar_wait(bar(Q_FULL), 0, abort_s, status);
+            if (tp) {
+                // tile i belongs to pipeline i & 1; its QK^T is issued two tiles ahead, right after the PV of tile i-2
+                for (int i = 0; ok && i < min(2, n_tiles); ++i) {
+                    ok = mbar_wait(bar(FULL + slot_of(2 * i)), par_of(2 * i), abort_s, status);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    qk(i, i);
+                    umma_commit(bar(S_FULL + i));
+                    umma_commit(bar(EMPTY + slot_of(2 * i)));
+                }
+                for (int i = 0; ok && i < n_tiles; ++i) {
+                    const int reg = i & 1, ph = (i >> 1) & 1;
+                    if (!mbar_wait(bar(FULL + slot_of(2 * i + 1)), par_of(2 * i + 1), abort_s, status)) break;
+                    if (!mbar_wait(bar(P_HALF + reg), ph, abort_s, status)) break;
+                    tc_fence_after_sync();
+                    pv(i, reg, 0);
+                    umma_commit(bar(PVH_DONE + reg));
+                    if (!mbar_wait(bar(P_FULL + reg), ph, abort_s, status)) break;
+                    tc_fence_after_sync();
+                    pv(i, reg, 1);
+                    umma_commit(bar(EMPTY + slot_of(2 * i + 1)));
+                    if (i + 2 < n_tiles) {
+                        if (!mbar_wait(bar(FULL + slot_of(2 * i + 4)), par_of(2 * i + 4), abort_s, status)) break;
+                        tc_fence_after_sync();
+                        qk(i + 2, reg);
+                        umma_commit(bar(S_FULL + reg));
+                        umma_commit(bar(EMPTY + slot_of(2 * i + 4)));
+                    }
+                }
+            } else {
             if (ok) ok = mbar_wait(bar(FULL + slot_of(0)), par_of(0), abort_s, status);
             if (ok) {
                 tc_fence_after_sync();
@@ -509,23 +546,26 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     umma_commit(bar(EMPTY + slot_of(2 * i + 2)));
                 }
             }
+            }
             umma_commit(bar(O_DONE));
         }
     } else {
         // ------------------------------------------------------------------ softmax warpgroups
         const int mt = warp >> 2, w4 = warp & 3;
-        if (mt < n_mt) {
+        if (mt < n_mt || tp) {
             const uint32_t lane_off = (uint32_t)(w4 * 32) << 16;
             const uint32_t tS = tmem_base + mt * 128 + lane_off, tO = tmem_base + 256 + mt * 128 + lane_off;
-            const int row = w4 * 32 + lane, grow = rg * 256 + mt * kTile + row;
-            const bool warp_has_rows = rg * 256 + mt * kTile + w4 * 32 < kv.M;
+            const int first = tp ? mt : 0, stride = tp ? 2 : 1;      // tiles of this warpgroup: first, first + stride, ...
+            const int row = w4 * 32 + lane, grow = rg * 256 + (tp ? 0 : mt * kTile) + row;
+            const bool warp_has_rows = rg * 256 + (tp ? 0 : mt * kTile) + w4 * 32 < kv.M;
             float m_used = -INFINITY, l = 0.f;
             float pend_m = 0.f;          // reference the row wants to move to at the start of its next tile
             bool pending = false;
             const uint64_t c2 = pack2(scale_log2, scale_log2);
             bool ok = true;
-            for (int i = 0; i < n_tiles; ++i) {
-                if (!__all_sync(0xffffffffu, mbar_wait(bar(S_FULL + mt), i & 1, abort_s, status))) { ok = false; break; }
+            for (int i = first; i < n_tiles; i += stride) {
+                const int ph = (tp ? i >> 1 : i) & 1;
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(S_FULL + mt), ph, abort_s, status))) { ok = false; break; }
                 tc_fence_after_sync();
                 const int valid = min(kTile, n_keys - i * kTile);
                 // Rescale O by f (rows that do not need it pass f = 1): no MMA touches this O between "S(i) complete"
@@ -543,7 +583,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     tmem_wait_st();
                 };
                 // a warp whose 32 rows all lie beyond M (row padding of the last M-tile) only takes part in the hand-offs
-                bool fast = i > 0 && valid == kTile, half_done = false;
+                bool fast = i > first && valid == kTile, half_done = false;
                 if (warp_has_rows && fast) {
                     // ---- common case: one sweep over S with the reference maximum carried over from earlier tiles.
                     // exp2(x - m_used) stays representable as long as x - m_used < 100, so the true maximum is only
@@ -604,7 +644,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                         if (__any_sync(0xffffffffu, mx > 100.f)) {
                             // A jump of more than 2^100 inside the tile (never seen in practice; kept for correctness):
                             // wait until the first half's PV has been accumulated, move the reference, redo keys 64-127.
-                            if (!__all_sync(0xffffffffu, mbar_wait(bar(PVH_DONE + mt), i & 1, abort_s, status))) { ok = false; break; }
+                            if (!__all_sync(0xffffffffu, mbar_wait(bar(PVH_DONE + mt), ph, abort_s, status))) { ok = false; break; }
                             tc_fence_after_sync();
                             float a0, a1, b0, b1;
                             unpack2(l2a, a0, a1);
@@ -668,7 +708,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     }
                     float target = mx * scale_log2;
                     if (pending) target = fmaxf(target, pend_m);
-                    if (i == 0) {
+                    if (i == first) {
                         m_used = target;
                     } else {
                         const bool need = pending || target > m_used + kRescaleThreshold;
@@ -705,7 +745,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     l += l0 + l1;
                 }
                 tmem_wait_st();
-                if (!SPARSE && valid != kTile && mt == 0) {
+                if (!SPARSE && valid != kTile && (tp || mt == 0)) {
                     // Last tile of the prefix: cache rows past the end may hold anything (even NaN patterns), and
                     // 0 * NaN would poison O.  Zero those V rows in shared memory before the PV MMA may start.
                     const int Lv = 2 * i + 1;
@@ -724,18 +764,53 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 if (!half_done) mbar_arrive_warp(bar(P_HALF + mt));
                 mbar_arrive_warp(bar(P_FULL + mt));
             }
+            // Tile-parity mode: warpgroup 1 publishes its (reference, sum) and is done; warpgroup 0 folds the second
+            // accumulator (same TMEM lanes, columns + 128) into its own while it writes the result.  The spare Q tile
+            // holds the published pairs.
+            float2 *pub = reinterpret_cast<float2 *>(q_s + kTileBytes);
+            const bool merge = tp && n_tiles > 1;
+            float w0 = 1.f, w1 = 0.f;
+            if (tp && mt == 1) {
+                if (ok && merge) {
+                    pub[row] = make_float2(m_used, l);
+                    __threadfence_block();
+                    mbar_arrive_warp(bar(PUB));
+                }
+                ok = false;                                  // nothing to write
+            }
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(O_DONE), 0, abort_s, status));
+            if (ok && merge) ok = __all_sync(0xffffffffu, mbar_wait(bar(PUB), 0, abort_s, status));
             if (ok) {
                 tc_fence_after_sync();
                 const bool row_ok = grow < kv.M;
+                if (merge) {
+                    const float2 o = pub[row];
+                    const float m_all = fmaxf(m_used, o.x);
+                    w0 = ex2(m_used - m_all);
+                    w1 = ex2(o.x - m_all);
+                    l = l * w0 + o.y * w1;
+                    m_used = m_all;
+                }
+                auto load_o = [&](int c0, uint32_t (&r)[32]) {
+                    tmem_ld32(tO + c0, r);
+                    if (merge) {
+                        uint32_t q[32];
+                        tmem_ld32(tO + 128 + c0, q);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            r[e] = __float_as_uint(fmaf(__uint_as_float(q[e]), w1, __uint_as_float(r[e]) * w0));
+                    } else {
+                        tmem_wait_ld();
+                    }
+                };
                 if (!SPARSE) {
                     const size_t item = (size_t)z * (plan.n_chunks + 1) + chunk;
                     float *po = ws + plan.off_part_o + (item * plan.Mw + grow) * kD;
 #pragma unroll
                     for (int c0 = 0; c0 < kD; c0 += 32) {
                         uint32_t r[32];
-                        tmem_ld32(tO + c0, r);
-                        tmem_wait_ld();
+                        load_o(c0, r);
                         if (row_ok) {
 #pragma unroll
                             for (int e = 0; e < 32; e += 4)
@@ -753,8 +828,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
 #pragma unroll
                     for (int c0 = 0; c0 < kD; c0 += 32) {
                         uint32_t r[32];
-                        tmem_ld32(tO + c0, r);
-                        tmem_wait_ld();
+                        load_o(c0, r);
                         if (row_ok) {
 #pragma unroll
                             for (int e = 0; e < 32; e += 4)
@@ -772,8 +846,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
 #pragma unroll
                     for (int c0 = 0; c0 < kD; c0 += 32) {
                         uint32_t r[32];
-                        tmem_ld32(tO + c0, r);
-                        tmem_wait_ld();
+                        load_o(c0, r);
                         if (row_ok) {
 #pragma unroll
                             for (int e = 0; e < 32; e += 8) {
