@@ -456,96 +456,115 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                                     q_row0 + mt * kTile + rb * 64);
             const uint32_t idesc_qk = idesc_bf16_f32(kTile, false, false);   // S[128 rows][128 keys]
             const uint32_t idesc_pv = idesc_bf16_f32(kD, false, true);       // O[128 rows][128 d], V is MN-major
-            const uint32_t q_addr = smem_u32(q_s);
-            // reg = which S/O region (and softmax warpgroup); the Q tile is reg with two M-tiles, tile 0 in tile-parity mode
-            auto qk = [&](int i, int reg) {
-                const uint32_t k_addr = smem_u32(kv_s + slot_of(2 * i) * kTileBytes);
-                const uint32_t qt = tp ? 0 : reg;
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t a = smem_desc_sw128(q_addr + qt * kTileBytes + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
-                    const uint64_t b = smem_desc_sw128(k_addr + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
-                    umma_ss(tmem_base + reg * 128, a, b, idesc_qk, ks > 0);
+            // The issuing thread runs in step with the tensor pipe (an MMA is accepted only as the previous one drains),
+            // so whatever it executes between two MMAs is idle time of the pipe.  Hence: shared-memory descriptors are
+            // a per-slot base plus a constant (same upper word for all of them: 1024-byte groups of eight rows, 128-byte
+            // swizzle); ring positions advance without divisions; operand waits are taken before a batch of MMAs, not
+            // inside it; the PV of a tile is issued in one go when P is already complete (half by half, with a commit
+            // between, only when the softmax is the slower side); and key/value slots are handed back to the producer
+            // by the softmax warpgroup that observes the next S (its commit covers every earlier MMA).
+            constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+            constexpr uint32_t kTileU = kTileBytes >> 4, kHalfU = kHalfBytes >> 4;     // 16-byte units
+            auto desc = [](uint32_t lo) { return ((uint64_t)kDescHi << 32) | lo; };
+            const uint32_t q_lo = ((smem_u32(q_s) >> 4) & 0x3FFFu) | (1u << 16);           // K-major: 16-byte leading offset
+            const uint32_t k_lo = ((smem_u32(kv_s) >> 4) & 0x3FFFu) | (1u << 16);
+            const uint32_t v_lo = ((smem_u32(kv_s) >> 4) & 0x3FFFu) | (kHalfU << 16);       // MN-major: the two d-halves
+            struct Ring {                                    // position of a load in the ring of slots, two loads per step
+                int slot;
+                uint32_t par;
+                __device__ void next() {
+                    slot += 2;
+                    if (slot >= kAttnSlots) { slot -= kAttnSlots; par ^= 1u; }
                 }
             };
-            auto pv = [&](int i, int mt, int half) {  // half 0: keys 0-63 of the tile, half 1: keys 64-127
-                const uint32_t v_addr = smem_u32(kv_s + slot_of(2 * i + 1) * kTileBytes);
+            auto ring_at = [](int L) { return Ring{L % kAttnSlots, (uint32_t)((L / kAttnSlots) & 1)}; };
+            // reg = which S/O region (and softmax warpgroup); the Q tile is reg with two M-tiles, tile 0 in tile-parity mode
+            auto qk = [&](int slot, int reg) {
+                const uint32_t a0 = q_lo + (tp ? 0u : (uint32_t)reg * kTileU), b0 = k_lo + (uint32_t)slot * kTileU;
 #pragma unroll
-                for (int ks = half * 4; ks < half * 4 + 4; ++ks) {      // 16 keys per step: 16 rows of 128 bytes in each d-half
-                    const uint64_t b = smem_desc_sw128(v_addr + ks * 2048, kHalfBytes, 1024);
-                    umma_ts(tmem_base + 256 + mt * 128, tmem_base + mt * 128 + ks * 8, b, idesc_pv, (i > (tp ? 1 : 0) || ks > 0) ? 1u : 0u);
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t off = (ks >> 2) * kHalfU + (ks & 3) * 2;
+                    umma_ss(tmem_base + reg * 128, desc(a0 + off), desc(b0 + off), idesc_qk, ks > 0);
                 }
+            };
+            // half 0: keys 0-63 of the tile, half 1: keys 64-127; 16 keys per step = 16 rows of 128 bytes in each d-half
+            auto pv = [&](int slot, int reg, int half, uint32_t acc) {
+                const uint32_t b0 = v_lo + (uint32_t)slot * kTileU;
+#pragma unroll
+                for (int ks = half * 4; ks < half * 4 + 4; ++ks)
+                    umma_ts(tmem_base + 256 + reg * 128, tmem_base + reg * 128 + ks * 8, desc(b0 + ks * (2048 >> 4)), idesc_pv, ks > 0 ? 1u : acc);
+            };
+            auto wait_full = [&](const Ring &r) { return mbar_wait(bar(FULL + r.slot), r.par, abort_s, status); };
+            auto pv_tile = [&](int slot, int reg, int ph, uint32_t acc) -> bool {
+                if (mbar_test_wait(bar(P_FULL + reg), ph)) {
+                    tc_fence_after_sync();
+                    pv(slot, reg, 0, acc);
+                    pv(slot, reg, 1, acc);
+                    return true;
+                }
+                if (!mbar_wait(bar(P_HALF + reg), ph, abort_s, status)) return false;
+                tc_fence_after_sync();
+                pv(slot, reg, 0, acc);
+                umma_commit(bar(PVH_DONE + reg));
+                if (!mbar_wait(bar(P_FULL + reg), ph, abort_s, status)) return false;
+                tc_fence_after_sync();
+                pv(slot, reg, 1, acc);
+                return true;
             };
             bool ok = mbar_wait(bar(Q_FULL), 0, abort_s, status);
             if (tp) {
                 // tile i belongs to pipeline i & 1; its QK^T is issued two tiles ahead, right after the PV of tile i-2
-                for (int i = 0; ok && i < min(2, n_tiles); ++i) {
-                    ok = mbar_wait(bar(FULL + slot_of(2 * i)), par_of(2 * i), abort_s, status);
+                Ring rk = ring_at(0), rv = ring_at(1);
+                for (int i = 0; ok && i < min(2, n_tiles); ++i, rk.next()) {
+                    ok = wait_full(rk);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    qk(i, i);
+                    qk(rk.slot, i);
                     umma_commit(bar(S_FULL + i));
-                    umma_commit(bar(EMPTY + slot_of(2 * i)));
                 }
-                for (int i = 0; ok && i < n_tiles; ++i) {
+                rk = ring_at(4);
+                for (int i = 0; ok && i < n_tiles; ++i, rk.next(), rv.next()) {
                     const int reg = i & 1, ph = (i >> 1) & 1;
-                    if (!mbar_wait(bar(FULL + slot_of(2 * i + 1)), par_of(2 * i + 1), abort_s, status)) break;
-                    if (!mbar_wait(bar(P_HALF + reg), ph, abort_s, status)) break;
-                    tc_fence_after_sync();
-                    pv(i, reg, 0);
-                    umma_commit(bar(PVH_DONE + reg));
-                    if (!mbar_wait(bar(P_FULL + reg), ph, abort_s, status)) break;
-                    tc_fence_after_sync();
-                    pv(i, reg, 1);
-                    umma_commit(bar(EMPTY + slot_of(2 * i + 1)));
+                    if (!wait_full(rv)) break;
+                    if (!pv_tile(rv.slot, reg, ph, i > 1 ? 1u : 0u)) break;
+                    // V(i) goes back by a commit of its own here: the next S of this pipeline needs K(i+2), and a gathering
+                    // producer posts K(i+2) only after it has issued two more loads, the first of them into V(i)'s slot
+                    umma_commit(bar(EMPTY + rv.slot));
                     if (i + 2 < n_tiles) {
-                        if (!mbar_wait(bar(FULL + slot_of(2 * i + 4)), par_of(2 * i + 4), abort_s, status)) break;
+                        if (!wait_full(rk)) break;
                         tc_fence_after_sync();
-                        qk(i + 2, reg);
+                        qk(rk.slot, reg);
                         umma_commit(bar(S_FULL + reg));
-                        umma_commit(bar(EMPTY + slot_of(2 * i + 4)));
                     }
                 }
             } else {
-            if (ok) ok = mbar_wait(bar(FULL + slot_of(0)), par_of(0), abort_s, status);
-            if (ok) {
-                tc_fence_after_sync();
-                qk(0, 0);
-                umma_commit(bar(S_FULL + 0));
-                if (n_mt == 2) { qk(0, 1); umma_commit(bar(S_FULL + 1)); }
-                umma_commit(bar(EMPTY + slot_of(0)));
-            }
-            for (int i = 0; ok && i < n_tiles; ++i) {
-                const bool more = i + 1 < n_tiles;
-                if (!mbar_wait(bar(FULL + slot_of(2 * i + 1)), par_of(2 * i + 1), abort_s, status)) break;
-                if (!mbar_wait(bar(P_HALF + 0), i & 1, abort_s, status)) break;
-                tc_fence_after_sync();
-                pv(i, 0, 0);
-                umma_commit(bar(PVH_DONE + 0));
-                if (!mbar_wait(bar(P_FULL + 0), i & 1, abort_s, status)) break;
-                tc_fence_after_sync();
-                pv(i, 0, 1);
-                if (more) {
-                    if (!mbar_wait(bar(FULL + slot_of(2 * i + 2)), par_of(2 * i + 2), abort_s, status)) break;
+                Ring rk = ring_at(0), rv = ring_at(1);
+                if (ok) ok = wait_full(rk);
+                if (ok) {
                     tc_fence_after_sync();
-                    qk(i + 1, 0);
+                    qk(rk.slot, 0);
                     umma_commit(bar(S_FULL + 0));
+                    qk(rk.slot, 1);
+                    umma_commit(bar(S_FULL + 1));
                 }
-                if (n_mt == 2) {
-                    if (!mbar_wait(bar(P_HALF + 1), i & 1, abort_s, status)) break;
-                    tc_fence_after_sync();
-                    pv(i, 1, 0);
-                    umma_commit(bar(PVH_DONE + 1));
-                    if (!mbar_wait(bar(P_FULL + 1), i & 1, abort_s, status)) break;
-                    tc_fence_after_sync();
-                    pv(i, 1, 1);
+                rk.next();
+                for (int i = 0; ok && i < n_tiles; ++i, rk.next(), rv.next()) {
+                    const bool more = i + 1 < n_tiles;
+                    const int ph = i & 1;
+                    const uint32_t acc = i > 0 ? 1u : 0u;
+                    if (!wait_full(rv)) break;
+                    if (more && !wait_full(rk)) break;
+                    if (!pv_tile(rv.slot, 0, ph, acc)) break;
+                    if (more) {
+                        qk(rk.slot, 0);
+                        umma_commit(bar(S_FULL + 0));
+                    }
+                    if (!pv_tile(rv.slot, 1, ph, acc)) break;
+                    if (more) {
+                        qk(rk.slot, 1);
+                        umma_commit(bar(S_FULL + 1));
+                    }
                 }
-                umma_commit(bar(EMPTY + slot_of(2 * i + 1)));
-                if (more) {
-                    if (n_mt == 2) { qk(i + 1, 1); umma_commit(bar(S_FULL + 1)); }
-                    umma_commit(bar(EMPTY + slot_of(2 * i + 2)));
-                }
-            }
             }
             umma_commit(bar(O_DONE));
         }
@@ -567,6 +586,14 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 const int ph = (tp ? i >> 1 : i) & 1;
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(S_FULL + mt), ph, abort_s, status))) { ok = false; break; }
                 tc_fence_after_sync();
+                // S(i) complete means every MMA issued before it is complete too: K(i) and (two M-tiles) V(i-1), whose PV
+                // was issued just before this QK^T, have been read for the last time; their slots go back to the producer.
+                if (w4 == 0 && lane == 0 && (tp || mt == 1)) {
+                    mbar_arrive(bar(EMPTY + slot_of(2 * i)));
+                    if (!tp && i >= 1) mbar_arrive(bar(EMPTY + slot_of(2 * i - 1)));
+                }
+                // phase of the "first half of PV accumulated" barrier before this tile's P exists (see the recovery path)
+                const uint32_t pvh_cur = mbar_test_wait(bar(PVH_DONE + mt), 0) ? 1u : 0u;
                 const int valid = min(kTile, n_keys - i * kTile);
                 // Rescale O by f (rows that do not need it pass f = 1): no MMA touches this O between "S(i) complete"
                 // (which implies PV(i-1) complete) and "P(i) ready".
@@ -644,7 +671,9 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                         if (__any_sync(0xffffffffu, mx > 100.f)) {
                             // A jump of more than 2^100 inside the tile (never seen in practice; kept for correctness):
                             // wait until the first half's PV has been accumulated, move the reference, redo keys 64-127.
-                            if (!__all_sync(0xffffffffu, mbar_wait(bar(PVH_DONE + mt), ph, abort_s, status))) { ok = false; break; }
+                            // (the issuing thread finds P incomplete, issues the first half and commits to this barrier,
+                            // which otherwise is not signalled at all: wait for the phase seen at the start of the tile)
+                            if (!__all_sync(0xffffffffu, mbar_wait(bar(PVH_DONE + mt), pvh_cur, abort_s, status))) { ok = false; break; }
                             tc_fence_after_sync();
                             float a0, a1, b0, b1;
                             unpack2(l2a, a0, a1);
