@@ -1,6 +1,7 @@
 // Host side of libmage: argument validation, workspace planning and kernel launches behind the C ABI.
 #include <algorithm>
 #include <atomic>
+#include <cmath>
 #include <cstdio>
 #include <mutex>
 
@@ -57,12 +58,23 @@ static Plan make_plan(const mage_kv_t *kv, int k_max = 0) {
     pl.Mw = (int)align_up(pl.M, 128);
     const int64_t heads = (int64_t)kv->P * kv->H_kv;
     const int64_t tiles_head = kv->N_max > 0 ? (kv->N_max + 127) / 128 : 1;
-    int64_t waves = heads * tiles_head / (148 * 32);
-    if (waves < 1) waves = 1;
-    if (waves > 12) waves = 12;
-    int64_t want = 148 * waves / heads - 1;               // the block's own keys take one more item per head
-    if (want > tiles_head) want = tiles_head;
-    if (want < 1) want = 1;
+    // Key chunks per head.  One CTA per (head, chunk) and one CTA per SM at a time, so the pass lasts
+    // about ceil(heads * c / 148) rounds of (tiles per chunk + a fixed start/finish cost of about four tile times); each
+    // chunk also costs a partial result written and merged.  Pick the c that minimises that estimate.  A paged pool
+    // usually holds sequences of different lengths, which N_max says nothing about: keep its chunks at most 64 tiles
+    // long so that the long sequences spread over many CTAs.
+    int64_t want = 1;
+    double best = 1e300;
+    const int64_t c_max = tiles_head < 148 ? tiles_head : 148;
+    for (int64_t c = 1; c <= c_max; ++c) {
+        const int64_t tiles_c = (tiles_head + c - 1) / c;
+        if (kv->page_size != 0 && tiles_c > 64 && c < c_max) continue;
+        // (the CTA for the block's own keys costs about five tile times and takes an SM like any other)
+        const double per_cta = (double)(tiles_c + 4), work = (double)(heads * c) * per_cta + 5.0 * (double)heads;
+        const double rounds = std::ceil(work / (148.0 * per_cta) - 1e-9);
+        const double cost = rounds * per_cta + 7.7e-5 * (double)heads * pl.M * (double)c;
+        if (cost < best) { best = cost; want = c; }
+    }
     int64_t len = kv->N_max > 0 ? (kv->N_max + want - 1) / want : 128;
     len = (int64_t)align_up((size_t)len, 128);
     pl.chunk_len = (int)len;
@@ -131,7 +143,7 @@ static mage_status exact_select_simt(const mage_kv_t *kv, const KvView &view, co
     if (tc::eligible(kv)) {
         tc::AttnMaps maps;
         auto kern_tc = tc::attn_kernel<false>;
-        if (tc::make_rows_map(&maps.q, q, (long long)kv->P * kv->H_q * kv->B) && tc::make_cache_map(&maps.k, kv, kv->k_cache) &&
+        if (tc::make_group_rows_map(&maps.q, q, (long long)kv->P * kv->H_kv, kv->H_q / kv->H_kv * kv->B) && tc::make_cache_map(&maps.k, kv, kv->k_cache) &&
             tc::make_cache_map(&maps.v, kv, kv->v_cache) && tc::make_rows_map(&maps.kb, k_blk, (long long)kv->P * kv->H_kv * kv->B) &&
             tc::make_rows_map(&maps.vb, v_blk, (long long)kv->P * kv->H_kv * kv->B) && opt_in_smem(kern_tc, tc::kAttnSmemBytesDense) == MAGE_OK) {
             dim3 tgrid(plan.n_chunks + 1, (view.M + 255) / 256, kv->P * kv->H_kv);
@@ -182,7 +194,7 @@ static mage_status sparse_simt(const mage_kv_t *kv, const KvView &view, const Pl
     if (!(kv->flags & MAGE_FLAG_SIMT_KERNELS) && tc::encode_fn() != nullptr) {
         tc::AttnMaps maps;
         auto kern_tc = tc::attn_kernel<true>;
-        if (tc::make_rows_map(&maps.q, q, (long long)kv->P * kv->H_q * kv->B) && opt_in_smem(kern_tc, tc::kAttnSmemBytesSparse) == MAGE_OK) {
+        if (tc::make_group_rows_map(&maps.q, q, (long long)kv->P * kv->H_kv, kv->H_q / kv->H_kv * kv->B) && opt_in_smem(kern_tc, tc::kAttnSmemBytesSparse) == MAGE_OK) {
             maps.k = maps.v = maps.kb = maps.vb = maps.q;     // unused by the gather producers
             const int n_rg = (view.M + 255) / 256, heads = kv->P * kv->H_kv;
             // few (head, row-group) pairs in the launch: split each head's keys over several CTAs and merge

@@ -42,6 +42,14 @@ inline bool make_rows_map(CUtensorMap *m, const void *base, long long rows) {
     return make_map(m, base, 2, dims, str);
 }
 
+// Queries as (d, G*B rows of one KV head, P*H_kv heads): a 128-row tile that reaches past the head's last query row
+// is filled with zeros there instead of the next head's rows (no work for the multipliers, nothing to mask later).
+inline bool make_group_rows_map(CUtensorMap *m, const void *base, long long groups, int rows_per_group) {
+    cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)rows_per_group, (cuuint64_t)groups};
+    cuuint64_t str[2] = {(cuuint64_t)kD * 2, (cuuint64_t)rows_per_group * kD * 2};
+    return make_map(m, base, 3, dims, str);
+}
+
 // The prefix cache as a rank-4 tensor: (d, N_max, H_kv, P) with the caller's strides, or (d, page_size, H_kv, num_pages).
 inline bool make_cache_map(CUtensorMap *m, const mage_kv_t *kv, const void *base) {
     if (kv->page_size == 0) {

@@ -447,13 +447,12 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
         // ------------------------------------------------------------------ MMA issue (one lane)
         if (lane == 0) {
             prefetch_tensormap(&maps.q);
-            const int q_row0 = (p * kv.H_q + h * kv.G) * kv.B + rg * 256;
             mbar_arrive_expect_tx(bar(Q_FULL), n_mt * kTileBytes);
             for (int mt = 0; mt < n_mt; ++mt)
                 for (int dh = 0; dh < 2; ++dh)
-                    for (int rb = 0; rb < 2; ++rb)
-                        tma_load_2d(smem_u32(q_s + mt * kTileBytes + dh * kHalfBytes + rb * kBoxBytes), &maps.q, bar(Q_FULL), dh * 64,
-                                    q_row0 + mt * kTile + rb * 64);
+                    for (int rb = 0; rb < 2; ++rb)     // (d, row within the KV head's G*B rows, head): rows past the head read as zeros
+                        tma_load_3d(smem_u32(q_s + mt * kTileBytes + dh * kHalfBytes + rb * kBoxBytes), &maps.q, bar(Q_FULL), dh * 64,
+                                    rg * 256 + mt * kTile + rb * 64, z);
             const uint32_t idesc_qk = idesc_bf16_f32(kTile, false, false);   // S[128 rows][128 keys]
             const uint32_t idesc_pv = idesc_bf16_f32(kD, false, true);       // O[128 rows][128 d], V is MN-major
             // The issuing thread runs in step with the tensor pipe (an MMA is accepted only as the previous one drains),
@@ -495,8 +494,12 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     umma_ts(tmem_base + 256 + reg * 128, tmem_base + reg * 128 + ks * 8, desc(b0 + ks * (2048 >> 4)), idesc_pv, ks > 0 ? 1u : acc);
             };
             auto wait_full = [&](const Ring &r) { return mbar_wait(bar(FULL + r.slot), r.par, abort_s, status); };
-            auto pv_tile = [&](int slot, int reg, int ph, uint32_t acc) -> bool {
-                if (mbar_test_wait(bar(P_FULL + reg), ph)) {
+            auto peek_p = [&](int reg, int ph) { return mbar_test_wait(bar(P_FULL + reg), ph); };
+            // Looks at barriers ahead of time: the test is issued before a batch of MMAs and its result is used after it,
+            // so its latency (about a hundred cycles even when the phase is complete) overlaps with the issue of the batch.
+            auto peek_full = [&](const Ring &r) { return mbar_test_wait(bar(FULL + r.slot), r.par); };
+            auto pv_tile = [&](int slot, int reg, int ph, uint32_t acc, bool p_ready) -> bool {
+                if (p_ready || mbar_test_wait(bar(P_FULL + reg), ph)) {
                     tc_fence_after_sync();
                     pv(slot, reg, 0, acc);
                     pv(slot, reg, 1, acc);
@@ -526,7 +529,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 for (int i = 0; ok && i < n_tiles; ++i, rk.next(), rv.next()) {
                     const int reg = i & 1, ph = (i >> 1) & 1;
                     if (!wait_full(rv)) break;
-                    if (!pv_tile(rv.slot, reg, ph, i > 1 ? 1u : 0u)) break;
+                    if (!pv_tile(rv.slot, reg, ph, i > 1 ? 1u : 0u, peek_p(reg, ph))) break;
                     // V(i) goes back by a commit of its own here: the next S of this pipeline needs K(i+2), and a gathering
                     // producer posts K(i+2) only after it has issued two more loads, the first of them into V(i)'s slot
                     umma_commit(bar(EMPTY + rv.slot));
@@ -548,19 +551,27 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     umma_commit(bar(S_FULL + 1));
                 }
                 rk.next();
+                bool v_ready = false, k_ready = false, p0_ready = false;          // looked at during the previous batch
                 for (int i = 0; ok && i < n_tiles; ++i, rk.next(), rv.next()) {
                     const bool more = i + 1 < n_tiles;
                     const int ph = i & 1;
                     const uint32_t acc = i > 0 ? 1u : 0u;
-                    if (!wait_full(rv)) break;
-                    if (more && !wait_full(rk)) break;
-                    if (!pv_tile(rv.slot, 0, ph, acc)) break;
+                    if (!v_ready && !wait_full(rv)) break;
+                    if (more && !k_ready && !wait_full(rk)) break;
+                    if (!pv_tile(rv.slot, 0, ph, acc, p0_ready)) break;
+                    const bool p1_ready = peek_p(1, ph);
                     if (more) {
                         qk(rk.slot, 0);
                         umma_commit(bar(S_FULL + 0));
                     }
-                    if (!pv_tile(rv.slot, 1, ph, acc)) break;
+                    if (!pv_tile(rv.slot, 1, ph, acc, p1_ready)) break;
                     if (more) {
+                        Ring rv1 = rv, rk1 = rk;
+                        rv1.next();
+                        rk1.next();
+                        v_ready = peek_full(rv1);
+                        k_ready = i + 2 < n_tiles && peek_full(rk1);
+                        p0_ready = peek_p(0, ph ^ 1);
                         qk(rk.slot, 1);
                         umma_commit(bar(S_FULL + 1));
                     }
