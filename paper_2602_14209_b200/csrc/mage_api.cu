@@ -166,7 +166,7 @@ static mage_status exact_select_simt(const mage_kv_t *kv, const KvView &view, co
         CUtensorMap map_q, map_k;
         if (tc::make_rows_map(&map_q, q, (long long)kv->P * kv->H_q * kv->B) && tc::make_cache_map(&map_k, kv, kv->k_cache) &&
             opt_in_smem(tc::score_kernel, tc::kScoreSmemBytes) == MAGE_OK) {
-            const int tpc = tc::tiles_per_cta_for((long long)kv->P * kv->H_kv, kv->N_max);
+            const int tpc = tc::tiles_per_cta_for((long long)kv->P * kv->H_kv, kv->N_max, kv->page_size != 0);
             const int tiles_head = (kv->N_max + tc::kTile - 1) / tc::kTile;
             dim3 sgrid((tiles_head + tpc - 1) / tpc, kv->P * kv->H_kv, 1);
             for (int r0 = 0; r0 < view.M; r0 += 256) {

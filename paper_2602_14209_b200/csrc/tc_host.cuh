@@ -71,14 +71,23 @@ inline bool eligible(const mage_kv_t *kv) {
     return encode_fn() != nullptr;
 }
 
-// Tiles per CTA so that the grid is a whole number of waves over 148 SMs with at most ~48 tiles per CTA.
-inline int tiles_per_cta_for(long long heads, int N_max) {
-    const long long tiles_head = (N_max + kTile - 1) / kTile, total = heads * tiles_head;
-    const long long waves = (total + 148LL * 48 - 1) / (148LL * 48);
-    long long tpc = (total + 148 * waves - 1) / (148 * waves);
-    if (tpc < 1) tpc = 1;
-    if (tpc > tiles_head) tpc = tiles_head;
-    return (int)tpc;
+// Key tiles per CTA of the score pass.  One CTA per SM at a time, so the pass lasts about ceil(heads * c / 148)
+// rounds of (tiles per CTA + a fixed start cost of about three tile times: the query tile, the row statistics, the
+// first key tile); take the number of pieces per head c that minimises that.  Paged pools (sequences of different
+// lengths) keep their pieces at most 64 tiles long.
+inline int tiles_per_cta_for(long long heads, int N_max, bool paged) {
+    const long long tiles_head = (N_max + kTile - 1) / kTile;
+    const long long c_max = tiles_head < 148 ? tiles_head : 148;
+    long long best_tpc = tiles_head > 0 ? tiles_head : 1;
+    double best = 1e300;
+    for (long long c = 1; c <= c_max; ++c) {
+        const long long tpc = (tiles_head + c - 1) / c;
+        if (paged && tpc > 64 && c < c_max) continue;
+        const long long rounds = (heads * c + 147) / 148;
+        const double cost = (double)rounds * (double)(tpc + 3);
+        if (cost < best) { best = cost; best_tpc = tpc; }
+    }
+    return (int)best_tpc;
 }
 
 }  // namespace tc
