@@ -158,6 +158,31 @@ def test_logit_jumps_beyond_the_lazy_rescale_range(oracle_mod, flags):
     assert abs(res["scores"][0, 0, 700] - 1.0) < 1e-5 and res["scores"][0, 0, :700].max() < 1e-30
 
 
+@pytest.mark.parametrize("H_q", [16, 28])
+def test_logit_jumps_inside_multi_tile_ctas(oracle_mod, H_q):
+    """The same jumps with enough (problem, head) pairs that a CTA of the exact pass walks several key tiles (a small
+    batch gets one tile per CTA and never carries a reference from tile to tile): the jump then arrives in the single-sweep
+    path, in the first half of a tile (redo on the careful path) and in the second half (the first half's PV has to be
+    accumulated before the reference moves).  H_q = 16: one M-tile per head (two pipelines over alternating tiles);
+    H_q = 28: two M-tiles."""
+    w = W.Workload("jumps_multi", H_q=H_q, H_kv=4, N=2048, B=32, k=512, T=2, P=40, n_heavy=8, seed=13)
+    batch = W.make_batch(w, device="cuda")
+    batch["q"][..., 0] = 16.0
+    batch["kc"][..., 0] = 0.0
+    batch["kb"][..., 0] = 0.0
+    # chunk 0 of a head is keys 0-1023: tile 2 first half, tile 3 second half, tile 5 first half, tile 6 second half
+    for j, val in ((300, 64.0), (450, 144.0), (700, 256.0), (860, 400.0)):
+        batch["kc"][:, 0, j, 0] = val
+    batch["kc"][:, 1, 1100, 0] = 192.0                             # head 1: second chunk, first tile
+    batch["kc"][:, 1, 1500, 0] = 200.0                             # ... and a moderate rise later in that chunk
+    batch["kc"][:, 2, 1990, 0] = 300.0                             # head 2: second half of the ragged-free last tile
+    res = H.run_gpu_block(batch, w)
+    assert res["status"] == 0
+    for p in (0, 39):
+        H.check_problem(oracle_mod, batch, res, w, p, check_topk=False, o_max_abs=2e-2)
+    assert abs(res["scores"][0, 0, 860] - 1.0) < 1e-5 and res["scores"][0, 0, :860].max() < 1e-30
+
+
 def test_layer_by_layer_runner_matches_batched_runner(oracle_mod):
     """pipeline.LayerwiseBlock (one launch per layer, P = 1 views of the same memory) against the batched call."""
     from paper_2602_14209_b200.pipeline import LayerwiseBlock
