@@ -400,12 +400,22 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             }
         } else {
             const int pt = tid - 256, cchunk = pt & 15, r0 = pt >> 4;
-            // Up to three gathers are in flight: the arrival for load L-2 is posted after load L has been issued.
+            // Up to three gathers are in flight and a load is posted (its FULL barrier signalled) once the two younger
+            // ones have been issued -- unless the ring is full: then everything in flight is waited for and posted before
+            // the warp blocks on the slot, so that the MMA side never waits for a load that has already landed.
             bool ok = true;
-            int issued = 0;
+            int issued = 0, posted = 0;
+            auto post_upto = [&](int n) {                 // loads [posted, n) have landed (the caller waited for them)
+                fence_proxy_async();
+                for (; posted < n; ++posted) mbar_arrive_warp(bar(FULL + slot_of(posted)));
+            };
             for (int L = 0; L < 2 * n_tiles && ok; ++L) {
                 const int i = L >> 1, is_v = L & 1, slot = slot_of(L);
-                if (!mbar_wait(bar(EMPTY + slot), par_of(L) ^ 1, abort_s, status)) { ok = false; break; }
+                if (!__all_sync(0xffffffffu, mbar_test_wait(bar(EMPTY + slot), par_of(L) ^ 1))) {
+                    cp_async_wait<0>();
+                    post_upto(issued);
+                    if (!mbar_wait(bar(EMPTY + slot), par_of(L) ^ 1, abort_s, status)) { ok = false; break; }
+                }
                 const __nv_bfloat16 *cache = is_v ? kv.v : kv.k, *blk = is_v ? v_blk : k_blk;
                 uint8_t *tile = kv_s + slot * kTileBytes + (cchunk >> 3) * kHalfBytes;
 #pragma unroll 4
@@ -424,24 +434,13 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 }
                 cp_async_commit();
                 issued = L + 1;
-                if (L >= 2) {
+                if (issued - posted > 2) {                // all but the two youngest groups are complete after this wait
                     cp_async_wait<2>();
-                    fence_proxy_async();
-                    mbar_arrive_warp(bar(FULL + slot_of(L - 2)));
+                    post_upto(issued - 2);
                 }
             }
-            if (ok) {
-                if (issued >= 2) {
-                    cp_async_wait<1>();
-                    fence_proxy_async();
-                    mbar_arrive_warp(bar(FULL + slot_of(issued - 2)));
-                }
-                cp_async_wait<0>();
-                fence_proxy_async();
-                mbar_arrive_warp(bar(FULL + slot_of(issued - 1)));
-            } else {
-                cp_async_wait<0>();
-            }
+            cp_async_wait<0>();
+            if (ok) post_upto(issued);
         }
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issue (one lane)
@@ -514,6 +513,9 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 pv(slot, reg, 1, acc);
                 return true;
             };
+            // The reuse step is a handful of tiles long and latency-bound: there the slots go back by commits right after
+            // their last MMA, which is sooner than the softmax warpgroup's wake-up.
+            constexpr bool kCommitFrees = SPARSE;
             bool ok = mbar_wait(bar(Q_FULL), 0, abort_s, status);
             if (tp) {
                 // tile i belongs to pipeline i & 1; its QK^T is issued two tiles ahead, right after the PV of tile i-2
@@ -524,6 +526,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     tc_fence_after_sync();
                     qk(rk.slot, i);
                     umma_commit(bar(S_FULL + i));
+                    if (kCommitFrees) umma_commit(bar(EMPTY + rk.slot));
                 }
                 rk = ring_at(4);
                 for (int i = 0; ok && i < n_tiles; ++i, rk.next(), rv.next()) {
@@ -538,6 +541,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                         tc_fence_after_sync();
                         qk(rk.slot, reg);
                         umma_commit(bar(S_FULL + reg));
+                        if (kCommitFrees) umma_commit(bar(EMPTY + rk.slot));
                     }
                 }
             } else {
@@ -549,6 +553,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     umma_commit(bar(S_FULL + 0));
                     qk(rk.slot, 1);
                     umma_commit(bar(S_FULL + 1));
+                    if (kCommitFrees) umma_commit(bar(EMPTY + rk.slot));
                 }
                 rk.next();
                 bool v_ready = false, k_ready = false, p0_ready = false;          // looked at during the previous batch
@@ -557,14 +562,20 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     const int ph = i & 1;
                     const uint32_t acc = i > 0 ? 1u : 0u;
                     if (!v_ready && !wait_full(rv)) break;
-                    if (more && !k_ready && !wait_full(rk)) break;
+                    // (a gathered K(i+1) may land after P(i) is ready: the reuse step does not hold PV(i) back for it)
+                    if (!SPARSE && more && !k_ready && !wait_full(rk)) break;
                     if (!pv_tile(rv.slot, 0, ph, acc, p0_ready)) break;
                     const bool p1_ready = peek_p(1, ph);
                     if (more) {
+                        if (SPARSE) {
+                            if (!wait_full(rk)) break;
+                            tc_fence_after_sync();
+                        }
                         qk(rk.slot, 0);
                         umma_commit(bar(S_FULL + 0));
                     }
                     if (!pv_tile(rv.slot, 1, ph, acc, p1_ready)) break;
+                    if (kCommitFrees) umma_commit(bar(EMPTY + rv.slot));
                     if (more) {
                         Ring rv1 = rv, rk1 = rk;
                         rv1.next();
@@ -574,6 +585,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                         p0_ready = peek_p(0, ph ^ 1);
                         qk(rk.slot, 1);
                         umma_commit(bar(S_FULL + 1));
+                        if (kCommitFrees) umma_commit(bar(EMPTY + rk.slot));
                     }
                 }
             }
@@ -599,7 +611,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 tc_fence_after_sync();
                 // S(i) complete means every MMA issued before it is complete too: K(i) and (two M-tiles) V(i-1), whose PV
                 // was issued just before this QK^T, have been read for the last time; their slots go back to the producer.
-                if (w4 == 0 && lane == 0 && (tp || mt == 1)) {
+                if (!SPARSE && w4 == 0 && lane == 0 && (tp || mt == 1)) {
                     mbar_arrive(bar(EMPTY + slot_of(2 * i)));
                     if (!tp && i >= 1) mbar_arrive(bar(EMPTY + slot_of(2 * i - 1)));
                 }
