@@ -621,7 +621,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 // Rescale O by f (rows that do not need it pass f = 1): no MMA touches this O between "S(i) complete"
                 // (which implies PV(i-1) complete) and "P(i) ready".
                 auto rescale_o = [&](float f) {
-#pragma unroll
+#pragma unroll 1
                     for (int c0 = 0; c0 < kD; c0 += 32) {
                         uint32_t r[32];
                         tmem_ld32(tO + c0, r);
@@ -744,7 +744,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     // ---- careful path (first tile, ragged last tile, or a jump of the maximum by more than 2^100):
                     // find the tile's maximum first, move the reference if it grew, then exponentiate.
                     float mx = -INFINITY;
-#pragma unroll
+#pragma unroll 1
                     for (int c0 = 0; c0 < kTile; c0 += 32) {
                         uint32_t r[32];
                         tmem_ld32(tS + c0, r);
@@ -775,7 +775,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     pending = false;
                     const float neg_m = -m_used;
                     float l0 = 0.f, l1 = 0.f;
-#pragma unroll
+#pragma unroll 1
                     for (int c0 = 0; c0 < kTile; c0 += 32) {
                         uint32_t r[32], pk[16];
                         tmem_ld32(tS + c0, r);
@@ -859,7 +859,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 if (!SPARSE) {
                     const size_t item = (size_t)z * (plan.n_chunks + 1) + chunk;
                     float *po = ws + plan.off_part_o + (item * plan.Mw + grow) * kD;
-#pragma unroll
+#pragma unroll 1
                     for (int c0 = 0; c0 < kD; c0 += 32) {
                         uint32_t r[32];
                         load_o(c0, r);
@@ -877,7 +877,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 } else if (gridDim.x > 1) {
                     const size_t item = (size_t)z * gridDim.x + chunk;
                     float *po = ws + plan.off_sparse_o + (item * plan.Mw + grow) * kD;
-#pragma unroll
+#pragma unroll 1
                     for (int c0 = 0; c0 < kD; c0 += 32) {
                         uint32_t r[32];
                         load_o(c0, r);
@@ -895,7 +895,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 } else {
                     const float inv = 1.f / l;
                     __nv_bfloat16 *po = out + ((long long)(p * kv.H_q + h * kv.G) * kv.B + grow) * kD;
-#pragma unroll
+#pragma unroll 1
                     for (int c0 = 0; c0 < kD; c0 += 32) {
                         uint32_t r[32];
                         load_o(c0, r);
