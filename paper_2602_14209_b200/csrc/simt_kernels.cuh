@@ -268,29 +268,57 @@ __global__ void __launch_bounds__(128) combine_kernel(KvView kv, Plan plan, floa
     const size_t item0 = (size_t)z * (plan.n_chunks + 1);
     const float *ml = ws + plan.off_part_ml;
     const float *po = ws + plan.off_part_o;
+    // Lane c % 32 owns chunk c's (m, l): all of them are loaded at once (up to kMaxPerLane per lane), the maximum and the
+    // sum are warp reductions in a fixed order, and the weights then travel by shuffle -- no chain of dependent loads.
+    constexpr int kMaxPerLane = 5;                       // 148 chunks per head at most
+    float m_c[kMaxPerLane], l_c[kMaxPerLane];
     float m_pre = -INFINITY;
-    for (int c = lane; c < nc; c += 32) m_pre = fmaxf(m_pre, ml[((item0 + c) * plan.Mw + r) * 2]);
+#pragma unroll
+    for (int u = 0; u < kMaxPerLane; ++u) {
+        const int c = lane + 32 * u;
+        m_c[u] = -INFINITY;
+        l_c[u] = 0.f;
+        if (c < nc) {
+            const float2 e = *reinterpret_cast<const float2 *>(ml + ((item0 + c) * plan.Mw + r) * 2);
+            m_c[u] = e.x;
+            l_c[u] = e.y;
+        }
+        m_pre = fmaxf(m_pre, m_c[u]);
+    }
 #pragma unroll
     for (int w = 16; w; w >>= 1) m_pre = fmaxf(m_pre, __shfl_xor_sync(0xffffffffu, m_pre, w));
     float l_pre = 0.f;
-    for (int c = 0; c < nc; ++c) {       // fixed order, identical on every lane
-        const float *e = ml + ((item0 + c) * plan.Mw + r) * 2;
-        l_pre += e[1] * exp2f(e[0] - m_pre);
-    }
+#pragma unroll
+    for (int u = 0; u < kMaxPerLane; ++u) l_pre += (lane + 32 * u < nc) ? l_c[u] * exp2f(m_c[u] - m_pre) : 0.f;
+#pragma unroll
+    for (int w = 16; w; w >>= 1) l_pre += __shfl_xor_sync(0xffffffffu, l_pre, w);
     if (lane == 0) ws[plan.off_neg_lse + (size_t)z * plan.Mw + r] = nc > 0 ? -(m_pre + log2f(l_pre)) : 0.f;
     const float *eb = ml + ((item0 + plan.n_chunks) * plan.Mw + r) * 2;
     const float m_blk = eb[0], l_blk = eb[1];
     const float m_all = fmaxf(m_pre, m_blk);
     const float w_blk = exp2f(m_blk - m_all);
-    float l_all = l_blk * w_blk;
+    const float l_all = l_blk * w_blk + (nc > 0 ? l_pre * exp2f(m_pre - m_all) : 0.f);
+    float w_c[kMaxPerLane];
+#pragma unroll
+    for (int u = 0; u < kMaxPerLane; ++u) w_c[u] = (lane + 32 * u < nc) ? exp2f(m_c[u] - m_all) : 0.f;
     float4 acc = *reinterpret_cast<const float4 *>(po + ((item0 + plan.n_chunks) * plan.Mw + r) * kD + lane * 4);
     acc.x *= w_blk; acc.y *= w_blk; acc.z *= w_blk; acc.w *= w_blk;
-    for (int c = 0; c < nc; ++c) {
-        const float *e = ml + ((item0 + c) * plan.Mw + r) * 2;
-        const float w = exp2f(e[0] - m_all);
-        l_all += e[1] * w;
-        const float4 v = *reinterpret_cast<const float4 *>(po + ((item0 + c) * plan.Mw + r) * kD + lane * 4);
-        acc.x = fmaf(v.x, w, acc.x); acc.y = fmaf(v.y, w, acc.y); acc.z = fmaf(v.z, w, acc.z); acc.w = fmaf(v.w, w, acc.w);
+#pragma unroll
+    for (int u = 0; u < kMaxPerLane; ++u) {
+        if (32 * u >= nc) break;
+        const int n_here = min(32, nc - 32 * u);
+        for (int c0 = 0; c0 < n_here; c0 += 4) {         // four independent 16-byte loads in flight per lane
+            float4 v[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                v[q] = c0 + q < n_here ? *reinterpret_cast<const float4 *>(po + ((item0 + 32 * u + c0 + q) * plan.Mw + r) * kD + lane * 4)
+                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {                // chunks in ascending order: the result does not depend on timing
+                const float w = __shfl_sync(0xffffffffu, w_c[u], (c0 + q) & 31);
+                acc.x = fmaf(v[q].x, w, acc.x); acc.y = fmaf(v[q].y, w, acc.y); acc.z = fmaf(v[q].z, w, acc.z); acc.w = fmaf(v[q].w, w, acc.w);
+            }
+        }
     }
     const float inv = 1.f / l_all;
     __nv_bfloat16 *dst = out + ((long long)(p * kv.H_q + h * kv.G) * kv.B + r) * kD + lane * 4;
