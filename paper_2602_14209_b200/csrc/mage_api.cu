@@ -195,7 +195,16 @@ static mage_status sparse_simt(const mage_kv_t *kv, const KvView &view, const Pl
         tc::AttnMaps maps;
         auto kern_tc = tc::attn_kernel<true>;
         if (tc::make_group_rows_map(&maps.q, q, (long long)kv->P * kv->H_kv, kv->H_q / kv->H_kv * kv->B) && opt_in_smem(kern_tc, tc::kAttnSmemBytesSparse) == MAGE_OK) {
-            maps.k = maps.v = maps.kb = maps.vb = maps.q;     // unused by the gather producers
+            maps.k = maps.v = maps.kb = maps.vb = maps.q;     // placeholders unless the TMA row gather below applies
+            long long c_rows = 0, c_pitch = 0;
+            const long long b_rows = (long long)kv->P * kv->H_kv * kv->B;
+            if (tc::eligible(kv) && tc::cache_as_rows(kv, &c_rows, &c_pitch) && tc::make_row_gather_map(&maps.k, kv->k_cache, c_rows, c_pitch) &&
+                tc::make_row_gather_map(&maps.v, kv->v_cache, c_rows, c_pitch) && tc::make_row_gather_map(&maps.kb, k_blk, b_rows, kD) &&
+                tc::make_row_gather_map(&maps.vb, v_blk, b_rows, kD) && !((reinterpret_cast<uintptr_t>(k_blk) | reinterpret_cast<uintptr_t>(v_blk)) & 15)) {
+                maps.gather_rows = (int)c_rows;
+                maps.gather_blk_rows = (int)b_rows;
+                maps.gather_pitch = (int)c_pitch;
+            }
             const int n_rg = (view.M + 255) / 256, heads = kv->P * kv->H_kv;
             // few (head, row-group) pairs in the launch: split each head's keys over several CTAs and merge
             int n_split = 1;

@@ -26,10 +26,11 @@ inline EncodeTiledFn encode_fn() {
 }
 
 // bf16 tensor of `rank` dims (dim 0 = the 128-element head dimension), boxes of 64 x 64 (x 1 x 1), 128-byte swizzle.
-inline bool make_map(CUtensorMap *m, const void *base, int rank, const cuuint64_t *dims, const cuuint64_t *strides_bytes) {
+inline bool make_map(CUtensorMap *m, const void *base, int rank, const cuuint64_t *dims, const cuuint64_t *strides_bytes,
+                     unsigned box_rows = 64) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    cuuint32_t box[4] = {64, 64, 1, 1}, estr[4] = {1, 1, 1, 1};
+    cuuint32_t box[4] = {64, box_rows, 1, 1}, estr[4] = {1, 1, 1, 1};
     if (dims[1] < 1) return false;
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), dims, strides_bytes, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -48,6 +49,26 @@ inline bool make_group_rows_map(CUtensorMap *m, const void *base, long long grou
     cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)rows_per_group, (cuuint64_t)groups};
     cuuint64_t str[2] = {(cuuint64_t)kD * 2, (cuuint64_t)rows_per_group * kD * 2};
     return make_map(m, base, 3, dims, str);
+}
+
+// Row gather of the reuse step: the same memory as a flat list of 256-byte rows with one pitch, fetched one row
+// (64 x 1 box per half) at a time; each row lands swizzled exactly as it would inside a 64-row box.
+inline bool make_row_gather_map(CUtensorMap *m, const void *base, long long rows, long long pitch_elems) {
+    if (rows < 1 || rows > 0x7fffffffLL) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)rows}, str[1] = {(cuuint64_t)pitch_elems * 2};
+    return make_map(m, base, 2, dims, str, 1);
+}
+// Number of rows and pitch of the cache seen that way; false when the strides do not form one pitch.
+inline bool cache_as_rows(const mage_kv_t *kv, long long *rows, long long *pitch) {
+    if (kv->page_size != 0) {
+        *rows = (long long)kv->num_pages * kv->H_kv * kv->page_size;
+        *pitch = kD;
+        return true;
+    }
+    if (kv->stride_n < kD || kv->stride_h % kv->stride_n || kv->stride_p % kv->stride_n) return false;
+    *pitch = kv->stride_n;
+    *rows = ((long long)(kv->P - 1) * kv->stride_p + (long long)(kv->H_kv - 1) * kv->stride_h) / kv->stride_n + kv->N_max;
+    return true;
 }
 
 // The prefix cache as a rank-4 tensor: (d, N_max, H_kv, P) with the caller's strides, or (d, page_size, H_kv, num_pages).

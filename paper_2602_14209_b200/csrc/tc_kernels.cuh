@@ -269,7 +269,11 @@ constexpr size_t kAttnSmemBytesDense = 1024 + kAttnQBytes + kAttnSlotsDense * kT
 constexpr size_t kAttnSmemBytesSparse = 1024 + kAttnQBytes + kAttnSlotsSparse * kTileBytes + 512 + kSparseTableCap * sizeof(int);
 constexpr float kRescaleThreshold = 8.f;               // log2 units
 
-struct AttnMaps { CUtensorMap q, k, v, kb, vb; };
+// gather_rows > 0 (reuse step only): k, v, kb, vb are flat row lists (pitch gather_pitch elements) with 64 x 1 boxes.
+struct AttnMaps {
+    CUtensorMap q, k, v, kb, vb;
+    int gather_rows = 0, gather_blk_rows = 0, gather_pitch = 0;
+};
 
 template <bool SPARSE>
 __global__ void __launch_bounds__(SPARSE ? 416 : 320, 1)
@@ -354,7 +358,8 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             return -1;
         }
         const long long off = cache_row_offset(kv, p, h, j, status);
-        return off < 0 ? -1 : (int)(off >> 3);
+        if (off < 0) return -1;
+        return maps.gather_rows > 0 ? (int)(off / maps.gather_pitch) : (int)(off >> 3);
     };
     const bool use_tab = SPARSE && n_cache <= kSparseTableCap;
     if (use_tab)
@@ -400,6 +405,43 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             }
         } else {
             const int pt = tid - 256, cchunk = pt & 15, r0 = pt >> 4;
+            if (maps.gather_rows > 0) {
+                // TMA row gather: thread r of the 128 producers fetches row r of every tile as two 64 x 1 boxes (the two
+                // d-halves).  Unlike 16-byte cp.async, these requests do not pass through the L1 miss queue, which
+                // limits a CTA to about 17 GB/s of scattered rows.  Rows that do not exist (a bad index, the tail of
+                // the last tile) are fetched from beyond the tensor and arrive as zeros.  Each warp announces its 32 rows
+                // (8 KB) on the slot's barrier before its lanes issue.
+                if (lane == 0) {
+                    prefetch_tensormap(&maps.k); prefetch_tensormap(&maps.v); prefetch_tensormap(&maps.kb); prefetch_tensormap(&maps.vb);
+                }
+                int issued = 0;
+                for (int L = 0; L < 2 * n_tiles; ++L) {
+                    const int i = L >> 1, is_v = L & 1, slot = slot_of(L);
+                    if (!__all_sync(0xffffffffu, mbar_wait(bar(EMPTY + slot), par_of(L) ^ 1, abort_s, status))) break;
+                    if (lane == 0) mbar_arrive_expect_tx(bar(FULL + slot), 32 * 256);
+                    __syncwarp();
+                    const int t = i * kTile + pt;
+                    const CUtensorMap *map = is_v ? &maps.v : &maps.k;
+                    int row = maps.gather_rows;                       // beyond the tensor: zero fill
+                    if (t < n_cache) {
+                        const int o = use_tab ? row_tab[t] : resolve(t);
+                        if (o >= 0) row = o;
+                    } else {
+                        map = is_v ? &maps.vb : &maps.kb;
+                        row = t < n_keys ? z * kv.B + (t - blk_shift) : maps.gather_blk_rows;
+                    }
+                    const uint32_t dst = smem_u32(kv_s + slot * kTileBytes + pt * 128);
+                    tma_load_2d(dst, map, bar(FULL + slot), 0, row);
+                    tma_load_2d(dst + kHalfBytes, map, bar(FULL + slot), 64, row);
+                    issued = L + 1;
+                }
+                if (*abort_s) {                                        // let the copies in flight land before the CTA leaves
+                    for (int L = max(0, issued - kAttnSlots); L < issued; ++L) {
+                        const long long t0 = clock64();
+                        while (!mbar_try_wait(bar(FULL + slot_of(L)), par_of(L)) && clock64() - t0 < 2000000) {}
+                    }
+                }
+            } else {
             // Up to three gathers are in flight and a load is posted (its FULL barrier signalled) once the two younger
             // ones have been issued -- unless the ring is full: then everything in flight is waited for and posted before
             // the warp blocks on the slot, so that the MMA side never waits for a load that has already landed.
@@ -441,6 +483,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             }
             cp_async_wait<0>();
             if (ok) post_upto(issued);
+            }
         }
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issue (one lane)
