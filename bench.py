@@ -260,50 +260,27 @@ def main():
     kb_h = [t.cpu().pin_memory() for t in kb_d]
     vb_h = [t.cpu().pin_memory() for t in vb_d]
     out_h = [torch.empty_like(o, device="cpu").pin_memory() for o in outs]
-    q_s, kb_s, vb_s = [torch.empty_like(t) for t in q_d], [torch.empty_like(t) for t in kb_d], [torch.empty_like(t) for t in vb_d]
-    h2d = sum(t.numel() * 2 for t in q_h + kb_h + vb_h)
-    d2h = sum(t.numel() * 2 for t in out_h)
 
-    # Copies run on their own streams so that step t+1's inputs arrive, and step t-1's output leaves, while step t
-    # computes; every byte still crosses PCIe inside the timed region and the block ends with all outputs on the host.
-    h2d_stream, d2h_stream = torch.cuda.Stream(), torch.cuda.Stream()
-    ev_in = [torch.cuda.Event() for _ in range(T)]
-    ev_out = [torch.cuda.Event() for _ in range(T)]
-    ev_free = torch.cuda.Event()
+    # pipeline.HostStagedBlocks: copies run on their own streams and two sets of staging buffers alternate, so block
+    # n+1's inputs arrive, and block n's outputs leave, while the other block computes; every byte still crosses PCIe
+    # inside the timed region and the region ends with all outputs on the host.
+    from paper_2602_14209_b200.pipeline import HostStagedBlocks
+    staged = HostStagedBlocks(ba, T)
+    h2d, d2h = staged.h2d_bytes(), staged.d2h_bytes()
 
     def e2e_block():
-        ev_free.record(main_stream)                      # staging buffers of the previous block are no longer read
-        h2d_stream.wait_event(ev_free)
-        with torch.cuda.stream(h2d_stream):
-            for t in range(T):
-                q_s[t].copy_(q_h[t], non_blocking=True); kb_s[t].copy_(kb_h[t], non_blocking=True); vb_s[t].copy_(vb_h[t], non_blocking=True)
-                ev_in[t].record(h2d_stream)
-        main_stream.wait_event(ev_in[0])
-        ba.exact_select(q_s[0], kb_s[0], vb_s[0], outs[0])
-        ba.select_async()
-        ev_out[0].record(main_stream)
-        if T > 1:
-            ba.join()
-        for t in range(1, T):
-            main_stream.wait_event(ev_in[t])
-            ba.sparse_step(q_s[t], kb_s[t], vb_s[t], outs[t])
-            ev_out[t].record(main_stream)
-        with torch.cuda.stream(d2h_stream):
-            for t in range(T):
-                d2h_stream.wait_event(ev_out[t])
-                out_h[t].copy_(outs[t], non_blocking=True)
-        main_stream.wait_stream(d2h_stream)
-        main_stream.wait_stream(ba.select_stream)
-        main_stream.synchronize()
+        staged.submit(q_h, kb_h, vb_h, out_h, main_stream)
 
     e2e_steps = args.steps
     for _ in range(min(args.warmup, 2)):
         e2e_block()
+    staged.finish(main_stream)
     barrier()
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     f0.record()
     for _ in range(e2e_steps):
         e2e_block()
+    staged.finish(main_stream)                       # the last block's outputs are on the host before the clock stops
     f1.record()
     barrier()
     e2e_ms_total = f0.elapsed_time(f1)

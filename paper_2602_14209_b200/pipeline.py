@@ -78,6 +78,75 @@ class BlockAttention:
         return res
 
 
+class HostStagedBlocks:
+    """Blocks whose per-step inputs live in pinned host memory and whose outputs go back to pinned host memory.
+
+    Two sets of device staging buffers alternate between consecutive blocks: the inputs of block n+1 cross PCIe while
+    block n computes, and the outputs of block n leave while block n+1 computes.  Nothing here waits on the host;
+    ``finish()`` does.  The prefix cache stays resident on the device (it is the state that block-level caching keeps).
+    """
+
+    def __init__(self, ba: BlockAttention, T: int, depth: int = 2):
+        kv, dev = ba.kv, ba.kv.device
+        self.ba, self.T, self.depth, self.n = ba, int(T), int(depth), 0
+        mk = lambda *shape: torch.empty(*shape, dtype=torch.bfloat16, device=dev)
+        self.q_s = [[mk(kv.P, kv.H_q, kv.B, kv.d) for _ in range(T)] for _ in range(depth)]
+        self.kb_s = [[mk(kv.P, kv.H_kv, kv.B, kv.d) for _ in range(T)] for _ in range(depth)]
+        self.vb_s = [[mk(kv.P, kv.H_kv, kv.B, kv.d) for _ in range(T)] for _ in range(depth)]
+        self.out_s = [[mk(kv.P, kv.H_q, kv.B, kv.d) for _ in range(T)] for _ in range(depth)]
+        self.h2d_stream, self.d2h_stream = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        self.ev_in = [[torch.cuda.Event() for _ in range(T)] for _ in range(depth)]
+        self.ev_out = [[torch.cuda.Event() for _ in range(T)] for _ in range(depth)]
+        self.ev_computed = [torch.cuda.Event() for _ in range(depth)]     # staging inputs of this set are no longer read
+        self.ev_drained = [torch.cuda.Event() for _ in range(depth)]      # staging outputs of this set are on the host
+
+    def h2d_bytes(self) -> int:
+        return sum(t.numel() * 2 for t in self.q_s[0] + self.kb_s[0] + self.vb_s[0])
+
+    def d2h_bytes(self) -> int:
+        return sum(t.numel() * 2 for t in self.out_s[0])
+
+    def submit(self, q_h: Sequence[torch.Tensor], kb_h, vb_h, out_h, main_stream=None):
+        """Enqueue one block; returns immediately.  ``out_h[t]`` is valid after ``finish()`` (or a sync on d2h_stream)."""
+        main = torch.cuda.current_stream() if main_stream is None else main_stream
+        b, T, ba = self.n % self.depth, self.T, self.ba
+        used_before = self.n >= self.depth
+        self.n += 1
+        if used_before:
+            self.h2d_stream.wait_event(self.ev_computed[b])
+        with torch.cuda.stream(self.h2d_stream):
+            for t in range(T):
+                self.q_s[b][t].copy_(q_h[t], non_blocking=True)
+                self.kb_s[b][t].copy_(kb_h[t], non_blocking=True)
+                self.vb_s[b][t].copy_(vb_h[t], non_blocking=True)
+                self.ev_in[b][t].record(self.h2d_stream)
+        if used_before:
+            main.wait_event(self.ev_drained[b])
+        with torch.cuda.stream(main):
+            main.wait_event(self.ev_in[b][0])
+            ba.exact_select(self.q_s[b][0], self.kb_s[b][0], self.vb_s[b][0], self.out_s[b][0])
+            ba.select_async(main)
+            self.ev_out[b][0].record(main)
+            if T > 1:
+                ba.join(main)
+            for t in range(1, T):
+                main.wait_event(self.ev_in[b][t])
+                ba.sparse_step(self.q_s[b][t], self.kb_s[b][t], self.vb_s[b][t], self.out_s[b][t])
+                self.ev_out[b][t].record(main)
+            self.ev_computed[b].record(main)
+        with torch.cuda.stream(self.d2h_stream):
+            for t in range(T):
+                self.d2h_stream.wait_event(self.ev_out[b][t])
+                out_h[t].copy_(self.out_s[b][t], non_blocking=True)
+            self.ev_drained[b].record(self.d2h_stream)
+
+    def finish(self, main_stream=None):
+        main = torch.cuda.current_stream() if main_stream is None else main_stream
+        main.wait_stream(self.d2h_stream)
+        main.wait_stream(self.ba.select_stream)
+        main.synchronize()
+
+
 class LayerwiseBlock:
     """One block of Algorithm 1 issued the way a model runs it: layer after layer.
 

@@ -218,3 +218,32 @@ def test_sparse_step_without_workspace_and_events_variant(oracle_mod):
     assert ev[0].elapsed_time(ev[3]) > 0 and ev[0].elapsed_time(ev[1]) > 0
     assert (out_a.float() - out_b.float()).abs().max() < 5e-3
     assert np.abs(out_b.float().cpu().numpy() - res["outs"][1]).max() < 5e-3
+
+
+def test_host_staged_blocks_match_the_resident_path(oracle_mod):
+    """pipeline.HostStagedBlocks (pinned host inputs and outputs, two alternating sets of staging buffers) over four
+    consecutive blocks with different inputs: every block's outputs on the host equal the resident-input run of that block."""
+    from paper_2602_14209_b200.pipeline import HostStagedBlocks
+    w = W.CONFIGS["cfg1_small"]
+    batch = W.make_batch(w, device="cuda")
+    res = H.run_gpu_block(batch, w)
+    ba, T = res["ba"], w.T
+    staged = HostStagedBlocks(ba, T)
+    host_out, expect = [], []
+    for blk in range(4):
+        scale = 1.0 + 0.25 * blk                                   # a different block each time
+        q = [(batch["q"][t].float() * scale).to(torch.bfloat16) for t in range(T)]
+        kb, vb = [batch["kb"][t] for t in range(T)], [batch["vb"][t] for t in range(T)]
+        direct = [torch.empty_like(ba.out) for _ in range(T)]
+        ba.run_block(q, kb, vb, direct)
+        torch.cuda.synchronize()
+        expect.append([o.cpu() for o in direct])
+        out_h = [torch.empty(ba.out.shape, dtype=torch.bfloat16).pin_memory() for _ in range(T)]
+        host_out.append(out_h)
+        staged.submit([t.cpu().pin_memory() for t in q], [t.cpu().pin_memory() for t in kb], [t.cpu().pin_memory() for t in vb], out_h)
+    staged.finish()
+    assert int(ba.status.item()) == 0
+    for blk in range(4):
+        for t in range(T):
+            assert torch.equal(host_out[blk][t], expect[blk][t]), (blk, t)
+    assert np.abs(expect[0][0].float().numpy() - res["outs"][0]).max() == 0.0
