@@ -40,23 +40,23 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *__restr
     }
 
     const bool vec_ok = (reinterpret_cast<uintptr_t>(s) & 15) == 0;
-    // Visit the row 8 elements per thread and iteration, all loads issued before any is used.
+    // Visit the row 16 elements per thread and iteration, all four 16-byte loads issued before any is used.
     auto for_each8 = [&](auto &&body) {
-        for (int base = 0; base < N; base += kTopkThreads * 8) {
-            float v[8];
+        for (int base = 0; base < N; base += kTopkThreads * 16) {
+            float v[16];
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                const int j = base + half * kTopkThreads * 4 + tid * 4;
+            for (int q4 = 0; q4 < 4; ++q4) {
+                const int j = base + q4 * kTopkThreads * 4 + tid * 4;
                 if (vec_ok && j + 3 < N) {
                     const float4 f = *reinterpret_cast<const float4 *>(s + j);
-                    v[half * 4 + 0] = f.x; v[half * 4 + 1] = f.y; v[half * 4 + 2] = f.z; v[half * 4 + 3] = f.w;
+                    v[q4 * 4 + 0] = f.x; v[q4 * 4 + 1] = f.y; v[q4 * 4 + 2] = f.z; v[q4 * 4 + 3] = f.w;
                 } else {
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) v[half * 4 + e] = j + e < N ? s[j + e] : 0.f;
+                    for (int e = 0; e < 4; ++e) v[q4 * 4 + e] = j + e < N ? s[j + e] : 0.f;
                 }
             }
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
+            for (int e = 0; e < 16; ++e) {
                 const int j = base + (e >> 2) * kTopkThreads * 4 + tid * 4 + (e & 3);
                 if (j < N) body(float_order_key(v[e]));
             }
@@ -122,7 +122,12 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *__restr
     }
     const unsigned T = prefix, need_eq = need;
 
-    unsigned run_gt = 0, run_eq = 0;
+    // Ordered emit.  A stretch of 32 x span entries at a time (span = 4096, less for short rows so that every warp has a
+    // share): warp w owns entries [w * span, (w + 1) * span) of the stretch, lane l the four entries at 128 * i + 4 * l of
+    // each of its span / 128 <= 32 rounds (coalesced 16-byte loads, eight in flight).  The
+    // scores are read once: each lane keeps one "greater" and one "equal" bit per entry (2 x 128 bits), the warps' counts
+    // meet in one block-wide prefix sum, and the positions are then written from the bit masks; rounds in which no lane of
+    // the warp holds a selected entry (almost all of them: k of N entries are selected) cost one ballot.
     auto load4 = [&](int j_first, float (&v)[4]) {
         if (vec_ok && j_first + 3 < N) {
             const float4 f = *reinterpret_cast<const float4 *>(s + j_first);
@@ -132,57 +137,76 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *__restr
             for (int e = 0; e < 4; ++e) v[e] = j_first + e < N ? s[j_first + e] : 0.f;
         }
     };
-    float nxt[4];
-    load4(tid * 4, nxt);
-    for (int base = 0; base < N; base += kTopkThreads * 4) {
-        const int j_first = base + tid * 4;
-        float v[4] = {nxt[0], nxt[1], nxt[2], nxt[3]};
-        if (base + kTopkThreads * 4 < N) load4(j_first + kTopkThreads * 4, nxt);     // prefetch the next chunk
-        unsigned gt = 0, eq = 0, is_gt = 0, is_eq = 0;
+    const int kWarpSpan = min(4096, ((N + 31) / 32 + 127) / 128 * 128), kStretch = 32 * kWarpSpan, rounds = kWarpSpan / 128;
+    unsigned run_gt = 0, run_eq = 0;                     // selected entries before the current stretch
+    for (int base = 0; base < N; base += kStretch) {
+        const int w0 = base + warp * kWarpSpan;
+        unsigned gt_bits[4] = {0, 0, 0, 0}, eq_bits[4] = {0, 0, 0, 0};
+        if (w0 < N) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            if (j_first + e < N) {
-                const unsigned key = float_order_key(v[e]);
-                if (key > T) { is_gt |= 1u << e; ++gt; }
-                else if (key == T) { is_eq |= 1u << e; ++eq; }
+            for (int i0 = 0; i0 < 32; i0 += 8) {
+                float v[8][4];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int j_first = w0 + (i0 + u) * 128 + lane * 4;
+                    if (i0 + u < rounds && j_first < N) load4(j_first, v[u]);
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int j_first = w0 + (i0 + u) * 128 + lane * 4;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        if (i0 + u < rounds && j_first + e < N) {
+                            const unsigned key = float_order_key(v[u][e]);
+                            if (key > T) gt_bits[i0 >> 3] |= 1u << (u * 4 + e);
+                            else if (key == T) eq_bits[i0 >> 3] |= 1u << (u * 4 + e);
+                        }
+                    }
+                }
             }
         }
-        const unsigned packed = (gt << 16) | eq;        // a chunk holds 4096 entries, so neither half overflows
-        unsigned incl = packed;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const unsigned up = __shfl_up_sync(0xffffffffu, incl, off);
-            if (lane >= off) incl += up;
-        }
-        if (lane == 31) warp_tot[warp] = incl;
+        unsigned n_gt = __popc(gt_bits[0]) + __popc(gt_bits[1]) + __popc(gt_bits[2]) + __popc(gt_bits[3]);
+        unsigned n_eq = __popc(eq_bits[0]) + __popc(eq_bits[1]) + __popc(eq_bits[2]) + __popc(eq_bits[3]);
+        n_gt = __reduce_add_sync(0xffffffffu, n_gt);
+        n_eq = __reduce_add_sync(0xffffffffu, n_eq);
+        if (lane == 0) { warp_tot[warp] = n_gt; hist[warp] = n_eq; }
         __syncthreads();
-        if (warp == 0) {
-            unsigned w = warp_tot[lane], wi = w;
+        // exclusive prefix of the warps' counts (every warp computes the one it needs) and the stretch totals
+        unsigned wg = warp_tot[lane], we = hist[lane];
+        unsigned gt_before = run_gt + __reduce_add_sync(0xffffffffu, lane < warp ? wg : 0u);
+        unsigned eq_before = run_eq + __reduce_add_sync(0xffffffffu, lane < warp ? we : 0u);
+        run_gt += __reduce_add_sync(0xffffffffu, wg);
+        run_eq += __reduce_add_sync(0xffffffffu, we);
+        if (n_gt + n_eq != 0) {
+#pragma unroll 1
+            for (int i = 0; i < rounds; ++i) {
+                const unsigned ng = (gt_bits[i >> 3] >> ((i & 7) * 4)) & 15u, ne = (eq_bits[i >> 3] >> ((i & 7) * 4)) & 15u;
+                if (__ballot_sync(0xffffffffu, (ng | ne) != 0u) == 0u) continue;
+                const unsigned packed = ((unsigned)__popc(ng) << 16) | (unsigned)__popc(ne);
+                unsigned incl = packed;
 #pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const unsigned up = __shfl_up_sync(0xffffffffu, wi, off);
-                if (lane >= off) wi += up;
+                for (int off = 1; off < 32; off <<= 1) {
+                    const unsigned up = __shfl_up_sync(0xffffffffu, incl, off);
+                    if (lane >= off) incl += up;
+                }
+                const unsigned tot = __shfl_sync(0xffffffffu, incl, 31), excl = incl - packed;
+                unsigned g = gt_before + (excl >> 16), q = eq_before + (excl & 0xffffu);
+                const int j_first = w0 + i * 128 + lane * 4;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (ng & (1u << e)) {
+                        out[g + min(q, need_eq)] = j_first + e;
+                        ++g;
+                    } else if (ne & (1u << e)) {
+                        if (q < need_eq) out[g + q] = j_first + e;
+                        ++q;
+                    }
+                }
+                gt_before += tot >> 16;
+                eq_before += tot & 0xffffu;
             }
-            warp_tot[lane] = wi - w;                    // exclusive prefix of the warp totals
-            if (lane == 31) suffix[0] = wi;             // chunk total
         }
-        __syncthreads();
-        const unsigned excl = incl - packed + warp_tot[warp];
-        unsigned gt_before = run_gt + (excl >> 16), eq_before = run_eq + (excl & 0xffffu);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            if (is_gt & (1u << e)) {
-                out[gt_before + min(eq_before, need_eq)] = j_first + e;
-                ++gt_before;
-            } else if (is_eq & (1u << e)) {
-                if (eq_before < need_eq) out[gt_before + eq_before] = j_first + e;
-                ++eq_before;
-            }
-        }
-        const unsigned tot = suffix[0];
-        run_gt += tot >> 16;
-        run_eq += tot & 0xffffu;
-        __syncthreads();
+        __syncthreads();                                  // warp_tot / hist are rewritten by the next stretch
     }
 }
 
