@@ -5,6 +5,7 @@
 // that issue TMA tile loads or gather rows with cp.async, and one warp that issues tcgen05.mma from a single lane
 // and owns the TMEM allocation.  All hand-offs go through mbarriers with bounded waits (sm100_ptx.cuh).
 #pragma once
+#include <type_traits>
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -207,16 +208,56 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                             if (c0 + e < n_cols) tail += ex2(fmaf(__uint_as_float(r[e]), scale_log2, neg_lse_s[col_lo + c0 + e]));
                     }
                 };
-                uint32_t ra[8], rb[8];
-                tmem_ld8(taddr, ra);
-                for (int c0 = 0; c0 < n_cols; c0 += 16) {
-                    tmem_wait_ld(ra);
-                    if (c0 + 8 < n_cols) tmem_ld8(taddr + c0 + 8, rb);
-                    step(ra, c0);
-                    if (c0 + 8 < n_cols) {
-                        tmem_wait_ld(rb);
-                        if (c0 + 16 < n_cols) tmem_ld8(taddr + c0 + 16, ra);
-                        step(rb, c0 + 8);
+                // The usual column counts (128, 64, and 112 = half of G*B = 224) run fully unrolled, 16 columns per step:
+                // no loop counters, compares or branches, constant offsets, half as many TMEM loads and waits.  The
+                // warps of this kernel issue more than half of all cycles, so instructions saved here are time saved.
+                auto step16 = [&](const uint32_t (&r)[16], int c0) {
+                    const float4 *nl4 = reinterpret_cast<const float4 *>(neg_lse_s + col_lo + c0);
+                    uint64_t x[8];
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        const float4 nq = nl4[q4];
+                        x[2 * q4] = fma2(pack2(__uint_as_float(r[4 * q4]), __uint_as_float(r[4 * q4 + 1])), c2, pack2(nq.x, nq.y));
+                        x[2 * q4 + 1] = fma2(pack2(__uint_as_float(r[4 * q4 + 2]), __uint_as_float(r[4 * q4 + 3])), c2, pack2(nq.z, nq.w));
+                    }
+                    ex2_mufu2_n(x);
+#pragma unroll
+                    for (int q = 0; q < 8; q += 2) { acc_a = add2(acc_a, x[q]); acc_b = add2(acc_b, x[q + 1]); }
+                };
+                auto sweep16 = [&](auto n_steps_tag) {
+                    constexpr int kSteps = decltype(n_steps_tag)::value;
+                    uint32_t ua[16], ub[16];
+                    tmem_ld16(taddr, ua);
+#pragma unroll
+                    for (int st = 0; st < kSteps; st += 2) {
+                        tmem_wait_ld(ua);
+                        if (st + 1 < kSteps) tmem_ld16(taddr + (st + 1) * 16, ub);
+                        step16(ua, st * 16);
+                        if (st + 1 < kSteps) {
+                            tmem_wait_ld(ub);
+                            if (st + 2 < kSteps) tmem_ld16(taddr + (st + 2) * 16, ua);
+                            step16(ub, (st + 1) * 16);
+                        }
+                    }
+                };
+                if (n_cols == 128) {
+                    sweep16(std::integral_constant<int, 8>{});
+                } else if (n_cols == 112) {
+                    sweep16(std::integral_constant<int, 7>{});
+                } else if (n_cols == 64) {
+                    sweep16(std::integral_constant<int, 4>{});
+                } else {
+                    uint32_t ra[8], rb[8];
+                    tmem_ld8(taddr, ra);
+                    for (int c0 = 0; c0 < n_cols; c0 += 16) {
+                        tmem_wait_ld(ra);
+                        if (c0 + 8 < n_cols) tmem_ld8(taddr + c0 + 8, rb);
+                        step(ra, c0);
+                        if (c0 + 8 < n_cols) {
+                            tmem_wait_ld(rb);
+                            if (c0 + 16 < n_cols) tmem_ld8(taddr + c0 + 16, ra);
+                            step(rb, c0 + 8);
+                        }
                     }
                 }
                 tc_fence_before_sync();
