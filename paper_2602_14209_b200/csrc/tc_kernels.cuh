@@ -739,7 +739,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                             const uint64_t x2 = fma2(pack2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1])), c2, neg_m2);
                             float x0, x1;
                             unpack2(x2, x0, x1);
-                            mx = fmaxf(mx, fmaxf(x0, x1));
+                            mx = max3(mx, x0, x1);
                             const float p0 = ex2(x0), p1 = ex2(x1);
                             if (e & 1) l2b = add2(l2b, pack2(p0, p1));
                             else l2a = add2(l2a, pack2(p0, p1));
