@@ -299,8 +299,11 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
 //
 // DENSE  (SPARSE = false): K/V tiles arrive by TMA from the cache (or from the block's own keys for the last
 //         chunk index); the result is the unnormalised partial (O, m, l) of the chunk, merged by combine_kernel.
-// SPARSE (SPARSE = true): four producer warps gather the k_eff selected cache rows (then the block's keys) with
-//         16-byte cp.async into the same swizzled layout; the result is the final bf16 output.
+// SPARSE (SPARSE = true): four producer warps gather the k_eff selected cache rows (then the block's keys) into the
+//         same swizzled layout -- one row per thread as two 64 x 1 TMA boxes when the cache has a single row pitch,
+//         16-byte cp.async otherwise; the result is the final bf16 output (or a partial one per CTA when a head's
+//         keys are split over several CTAs).
+// With a single M-tile (G*B <= 128) the two warpgroups take alternate key tiles of the same rows instead.
 // ------------------------------------------------------------------------------------------------------------
 constexpr int kAttnSlotsDense = 5;                     // ring of K/V tile slots: K(0) V(0) K(1) V(1) ...
 constexpr int kAttnSlotsSparse = 4;                    // one slot less: the room holds the gathered rows' offset table
