@@ -943,61 +943,66 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                         tmem_wait_ld();
                     }
                 };
+                // A thread holds a row of O, so a store straight from registers would put 16 bytes into each of 32
+                // different rows per instruction.  The rows go through shared memory instead (the key/value ring is idle
+                // now; 64 fp32 or 128 bf16 columns at a time, rows padded by 16 bytes against bank conflicts) and leave as
+                // whole 256-byte pieces, two rows per instruction.
+                constexpr int kStageRow = 256 + 16;
+                uint8_t *stg = kv_s + warp * (32 * kStageRow);
+                const int row0 = rg * 256 + (tp ? 0 : mt * kTile) + w4 * 32;              // first row of this warp
+                const int rows_ok = min(32, kv.M - row0);                                   // may be <= 0
+                auto flush = [&](uint8_t *dst_row0, size_t dst_pitch) {                     // 32 staged rows of 256 bytes -> global
+                    __syncwarp();
+#pragma unroll 4
+                    for (int it = 0; it < 16; ++it) {
+                        const int rr = it * 2 + (lane >> 4), cb = (lane & 15) * 16;
+                        const uint4 v = *reinterpret_cast<const uint4 *>(stg + rr * kStageRow + cb);
+                        if (rr < rows_ok) *reinterpret_cast<uint4 *>(dst_row0 + (size_t)rr * dst_pitch + cb) = v;
+                    }
+                    __syncwarp();
+                };
+                auto store_partial = [&](float *po_row0, float *pml_row) {                  // unnormalised O, then (m, l)
+#pragma unroll 1
+                    for (int c0 = 0; c0 < kD; c0 += 64) {
+#pragma unroll 1
+                        for (int c1 = 0; c1 < 64; c1 += 32) {
+                            uint32_t r[32];
+                            load_o(c0 + c1, r);
+#pragma unroll
+                            for (int e = 0; e < 32; e += 4)
+                                *reinterpret_cast<uint4 *>(stg + lane * kStageRow + (c1 + e) * 4) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
+                        }
+                        flush(reinterpret_cast<uint8_t *>(po_row0 + c0), (size_t)kD * 4);
+                    }
+                    if (row_ok) {
+                        pml_row[0] = m_used;
+                        pml_row[1] = l;
+                    }
+                };
                 if (!SPARSE) {
                     const size_t item = (size_t)z * (plan.n_chunks + 1) + chunk;
-                    float *po = ws + plan.off_part_o + (item * plan.Mw + grow) * kD;
-#pragma unroll 1
-                    for (int c0 = 0; c0 < kD; c0 += 32) {
-                        uint32_t r[32];
-                        load_o(c0, r);
-                        if (row_ok) {
-#pragma unroll
-                            for (int e = 0; e < 32; e += 4)
-                                *reinterpret_cast<uint4 *>(po + c0 + e) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
-                        }
-                    }
-                    if (row_ok) {
-                        float *pml = ws + plan.off_part_ml + (item * plan.Mw + grow) * 2;
-                        pml[0] = m_used;
-                        pml[1] = l;
-                    }
+                    store_partial(ws + plan.off_part_o + (item * plan.Mw + row0) * kD, ws + plan.off_part_ml + (item * plan.Mw + grow) * 2);
                 } else if (gridDim.x > 1) {
                     const size_t item = (size_t)z * gridDim.x + chunk;
-                    float *po = ws + plan.off_sparse_o + (item * plan.Mw + grow) * kD;
-#pragma unroll 1
-                    for (int c0 = 0; c0 < kD; c0 += 32) {
-                        uint32_t r[32];
-                        load_o(c0, r);
-                        if (row_ok) {
-#pragma unroll
-                            for (int e = 0; e < 32; e += 4)
-                                *reinterpret_cast<uint4 *>(po + c0 + e) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
-                        }
-                    }
-                    if (row_ok) {
-                        float *pml = ws + plan.off_sparse_ml + (item * plan.Mw + grow) * 2;
-                        pml[0] = m_used;
-                        pml[1] = l;
-                    }
+                    store_partial(ws + plan.off_sparse_o + (item * plan.Mw + row0) * kD, ws + plan.off_sparse_ml + (item * plan.Mw + grow) * 2);
                 } else {
                     const float inv = 1.f / l;
-                    __nv_bfloat16 *po = out + ((long long)(p * kv.H_q + h * kv.G) * kv.B + grow) * kD;
 #pragma unroll 1
                     for (int c0 = 0; c0 < kD; c0 += 32) {
                         uint32_t r[32];
                         load_o(c0, r);
-                        if (row_ok) {
 #pragma unroll
-                            for (int e = 0; e < 32; e += 8) {
-                                uint4 v;
-                                v.x = pack_bf16x2(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
-                                v.y = pack_bf16x2(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
-                                v.z = pack_bf16x2(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
-                                v.w = pack_bf16x2(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
-                                *reinterpret_cast<uint4 *>(po + c0 + e) = v;
-                            }
+                        for (int e = 0; e < 32; e += 8) {
+                            uint4 v;
+                            v.x = pack_bf16x2(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
+                            v.y = pack_bf16x2(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+                            v.z = pack_bf16x2(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
+                            v.w = pack_bf16x2(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
+                            *reinterpret_cast<uint4 *>(stg + lane * kStageRow + (c0 + e) * 2) = v;
                         }
                     }
+                    __nv_bfloat16 *po_row0 = out + ((long long)(p * kv.H_q + h * kv.G) * kv.B + row0) * kD;
+                    flush(reinterpret_cast<uint8_t *>(po_row0), (size_t)kD * 2);
                 }
             }
         }
