@@ -1023,16 +1023,33 @@ __global__ void __launch_bounds__(128) sparse_combine_kernel(KvView kv, Plan pla
     const int used = (tiles_all + per - 1) / per;               // splits that had work
     const float *ml = ws + plan.off_sparse_ml, *po = ws + plan.off_sparse_o;
     const size_t item0 = (size_t)z * n_split;
-    float m_all = -INFINITY;
-    for (int c = 0; c < used; ++c) m_all = fmaxf(m_all, ml[((item0 + c) * plan.Mw + r) * 2]);
-    float l_all = 0.f;
+    // lane c holds split c's (m, l) (at most 32 splits); maximum and sum are warp reductions in a fixed order, the weights
+    // travel by shuffle and four partial rows are in flight per lane
+    float m_c = -INFINITY, l_c = 0.f;
+    if (lane < used) {
+        const float2 e = *reinterpret_cast<const float2 *>(ml + ((item0 + lane) * plan.Mw + r) * 2);
+        m_c = e.x;
+        l_c = e.y;
+    }
+    float m_all = m_c;
+#pragma unroll
+    for (int w = 16; w; w >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xffffffffu, m_all, w));
+    const float w_c = lane < used ? exp2f(m_c - m_all) : 0.f;
+    float l_all = l_c * w_c;
+#pragma unroll
+    for (int w = 16; w; w >>= 1) l_all += __shfl_xor_sync(0xffffffffu, l_all, w);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int c = 0; c < used; ++c) {
-        const float *e = ml + ((item0 + c) * plan.Mw + r) * 2;
-        const float w = exp2f(e[0] - m_all);
-        l_all += e[1] * w;
-        const float4 v = *reinterpret_cast<const float4 *>(po + ((item0 + c) * plan.Mw + r) * kD + lane * 4);
-        acc.x = fmaf(v.x, w, acc.x); acc.y = fmaf(v.y, w, acc.y); acc.z = fmaf(v.z, w, acc.z); acc.w = fmaf(v.w, w, acc.w);
+    for (int c0 = 0; c0 < used; c0 += 4) {
+        float4 v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            v[q] = c0 + q < used ? *reinterpret_cast<const float4 *>(po + ((item0 + c0 + q) * plan.Mw + r) * kD + lane * 4)
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const float w = __shfl_sync(0xffffffffu, w_c, (c0 + q) & 31);
+            acc.x = fmaf(v[q].x, w, acc.x); acc.y = fmaf(v[q].y, w, acc.y); acc.z = fmaf(v[q].z, w, acc.z); acc.w = fmaf(v[q].w, w, acc.w);
+        }
     }
     const float inv = 1.f / l_all;
     __nv_bfloat16 *dst = out + ((long long)(p * kv.H_q + h * kv.G) * kv.B + r) * kD + lane * 4;
