@@ -96,6 +96,25 @@ static Plan make_plan(const mage_kv_t *kv, int k_max = 0) {
     return pl;
 }
 
+// Launch with the programmatic-serialization attribute: the kernel may be scheduled while its predecessor in the stream is
+// still running; every kernel launched this way begins with griddepcontrol.wait, so it touches no global memory before
+// the predecessor has completed.  What is saved is the launch gap between dependent kernels (a few microseconds each,
+// which is most of a single-layer reuse step).
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 static mage_status launch_check() {
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
@@ -147,7 +166,8 @@ static mage_status exact_select_simt(const mage_kv_t *kv, const KvView &view, co
             tc::make_cache_map(&maps.v, kv, kv->v_cache) && tc::make_rows_map(&maps.kb, k_blk, (long long)kv->P * kv->H_kv * kv->B) &&
             tc::make_rows_map(&maps.vb, v_blk, (long long)kv->P * kv->H_kv * kv->B) && opt_in_smem(kern_tc, tc::kAttnSmemBytesDense) == MAGE_OK) {
             dim3 tgrid(plan.n_chunks + 1, (view.M + 255) / 256, kv->P * kv->H_kv);
-            kern_tc<<<tgrid, 320, tc::kAttnSmemBytesDense, st>>>(maps, view, plan, k_blk, v_blk, nullptr, nullptr, 0, scale_log2, ws, nullptr, dev_status);
+            launch_pdl(kern_tc, tgrid, dim3(320), tc::kAttnSmemBytesDense, st, maps, view, plan, k_blk, v_blk, (const int *)nullptr, (const int *)nullptr, 0, scale_log2, ws,
+                       (__nv_bfloat16 *)nullptr, dev_status);
             if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
             tc_attn_done = true;
         }
@@ -158,7 +178,7 @@ static mage_status exact_select_simt(const mage_kv_t *kv, const KvView &view, co
     }
     if (ev) cudaEventRecord(ev[1], st);
     const int rows_total = kv->P * kv->H_kv * view.M;
-    combine_kernel<<<(rows_total + 3) / 4, 128, 0, st>>>(view, plan, ws, out);
+    launch_pdl(combine_kernel, dim3((rows_total + 3) / 4), dim3(128), 0, st, view, plan, ws, out);
     if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
     if (ev) cudaEventRecord(ev[2], st);
     bool tc_score_done = false;
@@ -170,8 +190,8 @@ static mage_status exact_select_simt(const mage_kv_t *kv, const KvView &view, co
             const int tiles_head = (kv->N_max + tc::kTile - 1) / tc::kTile;
             dim3 sgrid((tiles_head + tpc - 1) / tpc, kv->P * kv->H_kv, 1);
             for (int r0 = 0; r0 < view.M; r0 += 256) {
-                tc::score_kernel<<<sgrid, tc::kScoreThreads, tc::kScoreSmemBytes, st>>>(map_q, map_k, view, plan, r0, std::min(256, view.M - r0),
-                                                                                       tpc, scale_log2, ws, scores, r0 > 0, dev_status);
+                launch_pdl(tc::score_kernel, sgrid, dim3(tc::kScoreThreads), tc::kScoreSmemBytes, st, map_q, map_k, view, plan, r0, std::min(256, view.M - r0),
+                           tpc, scale_log2, (const float *)ws, scores, (int)(r0 > 0), dev_status);
                 if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
             }
             tc_score_done = true;
@@ -216,11 +236,11 @@ static mage_status sparse_simt(const mage_kv_t *kv, const KvView &view, const Pl
                 if (n_split < 1) n_split = 1;
             }
             dim3 tgrid(n_split, n_rg, heads);
-            kern_tc<<<tgrid, 416, tc::kAttnSmemBytesSparse, st>>>(maps, view, plan, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, ws, out, dev_status);
+            launch_pdl(kern_tc, tgrid, dim3(416), tc::kAttnSmemBytesSparse, st, maps, view, plan, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, ws, out, dev_status);
             if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
             if (n_split > 1) {
                 const int rows_total = heads * view.M;
-                tc::sparse_combine_kernel<<<(rows_total + 3) / 4, 128, 0, st>>>(view, plan, n_split, k, k_eff, ws, out);
+                launch_pdl(tc::sparse_combine_kernel, dim3((rows_total + 3) / 4), dim3(128), 0, st, view, plan, n_split, k, k_eff, (const float *)ws, out);
                 return launch_check();
             }
             return MAGE_OK;

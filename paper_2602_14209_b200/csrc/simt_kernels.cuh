@@ -259,6 +259,10 @@ __global__ void __launch_bounds__(kThreads) score_kernel(KvView kv, Plan plan, c
 //  - prefix chunks + the block's own keys -> normalised bf16 output.
 __global__ void __launch_bounds__(128) combine_kernel(KvView kv, Plan plan, float *__restrict__ ws,
                                                       __nv_bfloat16 *__restrict__ out) {
+    // may have been launched while the attention kernel was still running (programmatic dependent launch): wait for it,
+    // then let the score kernel's CTAs be scheduled
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     const int rows_total = kv.P * kv.H_kv * kv.M;
     if (warp >= rows_total) return;

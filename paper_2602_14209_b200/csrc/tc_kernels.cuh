@@ -63,6 +63,8 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
              int row_begin, int rows, int tiles_per_cta, float scale_log2, const float *__restrict__ ws,
              float *__restrict__ scores, int accumulate, unsigned *status) {
     using namespace ptx;
+    pdl_wait();
+    pdl_launch_dependents();
     const int z = blockIdx.y, p = z / kv.H_kv, h = z % kv.H_kv;
     const int N = seq_len_of(kv, p);
     const int tiles_total = (N + kTile - 1) / kTile;
@@ -325,6 +327,8 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             const __nv_bfloat16 *__restrict__ v_blk, const int *__restrict__ indices, const int *__restrict__ k_eff_arr, int k,
             float scale_log2, float *__restrict__ ws, __nv_bfloat16 *__restrict__ out, unsigned *status) {
     using namespace ptx;
+    pdl_wait();                      // everything below may read what the previous kernel in the stream wrote
+    pdl_launch_dependents();
     constexpr int kMmaWarp = SPARSE ? 12 : 9;
     constexpr int kAttnSlots = SPARSE ? kAttnSlotsSparse : kAttnSlotsDense;
     const int chunk = blockIdx.x, rg = blockIdx.y, z = blockIdx.z, p = z / kv.H_kv, h = z % kv.H_kv;
@@ -1015,6 +1019,8 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
 // Merge of a reuse step that was split over n_split CTAs per KV head: one warp per query row, fixed order.
 __global__ void __launch_bounds__(128) sparse_combine_kernel(KvView kv, Plan plan, int n_split, int k, const int *__restrict__ k_eff_arr,
                                                              const float *__restrict__ ws, __nv_bfloat16 *__restrict__ out) {
+    ptx::pdl_wait();
+    ptx::pdl_launch_dependents();
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (warp >= kv.P * kv.H_kv * kv.M) return;
     const int z = warp / kv.M, r = warp % kv.M, p = z / kv.H_kv, h = z % kv.H_kv;
