@@ -97,17 +97,26 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *__restr
                 if ((key & mask) == prefix) atomicAdd(&hist[(key >> lo) & dmask], 1u);
             });
             __syncthreads();
-            // suffix[t] = number of candidates whose digit is >= t
-            if (tid < 256) suffix[tid] = hist[tid];
+            // suffix[t] = number of candidates whose digit is >= t: warps 0-7 scan 32 bins each from the top down with
+            // shuffles, then add the totals of the warps above them (two barriers instead of sixteen)
+            if (tid < 256) {
+                unsigned v = hist[tid];
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const unsigned dn = __shfl_down_sync(0xffffffffu, v, off);
+                    if (lane + off < 32) v += dn;
+                }
+                suffix[tid] = v;                                   // inclusive suffix sum inside the warp's 32 bins
+                if (lane == 0) warp_tot[warp] = v;                 // total of bins [32 * warp, 32 * warp + 32)
+            }
             if (tid == 0) suffix[256] = 0;
             __syncthreads();
-            for (int off = 1; off < 256; off <<= 1) {
-                unsigned add = 0;
-                if (tid < 256 && tid + off < 256) add = suffix[tid + off];
-                __syncthreads();
-                if (tid < 256) suffix[tid] += add;
-                __syncthreads();
+            if (tid < 256) {
+                unsigned above = 0;
+                for (int w = warp + 1; w < 8; ++w) above += warp_tot[w];
+                suffix[tid] += above;
             }
+            __syncthreads();
             if (tid < 256 && suffix[tid] >= need && suffix[tid + 1] < need) {
                 sel_digit = tid;
                 sel_need = need - suffix[tid + 1];
