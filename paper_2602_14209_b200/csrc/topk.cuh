@@ -13,15 +13,15 @@ __device__ __forceinline__ unsigned float_order_key(float f) {
 }
 
 // One CTA per (problem, KV head).
-//  1. a min/max pass finds the keys' common leading bits; radix passes of up to 8 bits over the remaining bits
-//     find the k_eff-th largest key T and how many entries equal to T are still needed (shared-memory histograms);
+//  1. three radix passes (11 + 11 + 10 key bits from the top, shared-memory histograms) find the k_eff-th largest key T
+//     and how many entries equal to T are still needed;
 //  2. one ordered pass emits every position with key > T and the first `need_eq` positions with key == T,
 //     placed by a block-wide prefix sum, so the output is ascending and ties go to the smaller position.
 __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *__restrict__ scores,
                                                             const int *__restrict__ seq_lens, int H_kv, int N_max,
                                                             int k, int *__restrict__ indices, int *__restrict__ k_eff_out) {
-    __shared__ unsigned hist[256];
-    __shared__ unsigned suffix[257];
+    __shared__ unsigned hist4[4][2048];
+    __shared__ unsigned hist[32];
     __shared__ unsigned warp_tot[32];
     __shared__ unsigned sel_digit, sel_need;
 
@@ -63,71 +63,45 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *__restr
         }
     };
 
-    // Pass 0: smallest and largest key.  Their common leading bits need no radix pass (block scores of one head
-    // usually share sign, exponent and a few mantissa bits), and a constant row is decided here.
-    unsigned kmin = 0xffffffffu, kmax = 0u;
-    for_each8([&](unsigned key) { kmin = min(kmin, key); kmax = max(kmax, key); });
-    kmin = __reduce_min_sync(0xffffffffu, kmin);
-    kmax = __reduce_max_sync(0xffffffffu, kmax);
-    if (lane == 0) { warp_tot[warp] = kmin; hist[warp] = kmax; }
-    __syncthreads();
-    if (warp == 0) {
-        kmin = __reduce_min_sync(0xffffffffu, warp_tot[lane]);
-        kmax = __reduce_max_sync(0xffffffffu, hist[lane]);
-        if (lane == 0) { suffix[0] = kmin; suffix[1] = kmax; }
-    }
-    __syncthreads();
-    kmin = suffix[0];
-    kmax = suffix[1];
-    __syncthreads();
-
-    unsigned prefix = kmax, mask = 0xffffffffu, need = (unsigned)k_eff;
-    if (kmin != kmax) {
-        int hi = 31 - __clz(kmin ^ kmax);                 // highest bit in which any two keys differ
-        mask = hi == 31 ? 0u : ~((2u << hi) - 1u);
-        prefix = kmax & mask;
-        // Radix passes of up to 8 bits from there down.  Only keys that still match the prefix touch the
-        // histogram, so after the first pass the shared-memory atomics are few.
-        while (hi >= 0) {
-            const int lo = hi >= 7 ? hi - 7 : 0;
-            const unsigned dmask = (1u << (hi - lo + 1)) - 1u;
-            if (tid < 256) hist[tid] = 0;
-            __syncthreads();
-            for_each8([&](unsigned key) {
-                if ((key & mask) == prefix) atomicAdd(&hist[(key >> lo) & dmask], 1u);
-            });
-            __syncthreads();
-            // suffix[t] = number of candidates whose digit is >= t: warps 0-7 scan 32 bins each from the top down with
-            // shuffles, then add the totals of the warps above them (two barriers instead of sixteen)
-            if (tid < 256) {
-                unsigned v = hist[tid];
+    // Three radix passes over the 32 key bits, 11 + 11 + 10 bits from the top: each reads the row once (the launch is bound
+    // by L2 bandwidth times the number of passes, so fewer, wider digits beat a min/max pre-pass plus 8-bit digits).  Keys of
+    // one head crowd into a few values of the first digit (same sign, neighbouring exponents), so the histogram is kept
+    // in four copies (warp & 3) to spread the shared-memory atomics; after the first pass only keys that match the prefix
+    // found so far touch it.
+    unsigned prefix = 0u, mask = 0u, need = (unsigned)k_eff;
+#pragma unroll 1
+    for (int pass = 0; pass < 3; ++pass) {
+        const int lo = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+        const unsigned dmask = pass == 2 ? 1023u : 2047u;
+        for (int t = tid; t < 4 * 2048; t += kTopkThreads) (&hist4[0][0])[t] = 0;
+        __syncthreads();
+        unsigned *my_hist = hist4[warp & 3];
+        for_each8([&](unsigned key) {
+            if ((key & mask) == prefix) atomicAdd(&my_hist[(key >> lo) & dmask], 1u);
+        });
+        __syncthreads();
+        // number of candidates with digit >= d, for the two digits 2 * tid and 2 * tid + 1 of this thread: suffix sums by
+        // shuffles inside the warp (64 digits), then the totals of the warps above
+        const unsigned c0 = hist4[0][2 * tid] + hist4[1][2 * tid] + hist4[2][2 * tid] + hist4[3][2 * tid];
+        const unsigned c1 = hist4[0][2 * tid + 1] + hist4[1][2 * tid + 1] + hist4[2][2 * tid + 1] + hist4[3][2 * tid + 1];
+        unsigned v = c0 + c1;
 #pragma unroll
-                for (int off = 1; off < 32; off <<= 1) {
-                    const unsigned dn = __shfl_down_sync(0xffffffffu, v, off);
-                    if (lane + off < 32) v += dn;
-                }
-                suffix[tid] = v;                                   // inclusive suffix sum inside the warp's 32 bins
-                if (lane == 0) warp_tot[warp] = v;                 // total of bins [32 * warp, 32 * warp + 32)
-            }
-            if (tid == 0) suffix[256] = 0;
-            __syncthreads();
-            if (tid < 256) {
-                unsigned above = 0;
-                for (int w = warp + 1; w < 8; ++w) above += warp_tot[w];
-                suffix[tid] += above;
-            }
-            __syncthreads();
-            if (tid < 256 && suffix[tid] >= need && suffix[tid + 1] < need) {
-                sel_digit = tid;
-                sel_need = need - suffix[tid + 1];
-            }
-            __syncthreads();
-            prefix |= sel_digit << lo;
-            mask |= dmask << lo;
-            need = sel_need;
-            __syncthreads();
-            hi = lo - 1;
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned dn = __shfl_down_sync(0xffffffffu, v, off);
+            if (lane + off < 32) v += dn;
         }
+        if (lane == 0) warp_tot[warp] = v;
+        __syncthreads();
+        unsigned above = 0;
+        for (int w = warp + 1; w < 32; ++w) above += warp_tot[w];
+        const unsigned ge0 = v + above, ge1 = ge0 - c0, ge2 = ge1 - c1;       // candidates with digit >= 2t, >= 2t+1, >= 2t+2
+        if (ge1 >= need && ge2 < need) { sel_digit = 2 * tid + 1; sel_need = need - ge2; }
+        else if (ge0 >= need && ge1 < need) { sel_digit = 2 * tid; sel_need = need - ge1; }
+        __syncthreads();
+        prefix |= sel_digit << lo;
+        mask |= dmask << lo;
+        need = sel_need;
+        __syncthreads();
     }
     const unsigned T = prefix, need_eq = need;
 

@@ -111,6 +111,28 @@ def test_topk_edge_cases_against_full_sort():
             assert (got[len(ref):] == -1).all()
 
 
+def test_topk_long_rows_negative_values_and_quantised_ties():
+    """Rows longer than one emit stretch (32 warps x 4096 entries), values of both signs, and a row quantised to 64 levels so
+    that the threshold value has thousands of ties: positions come out ascending with ties to the smaller position."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(7)
+    P, H_kv, N_max, k = 2, 2, 300001, 1000
+    sc = torch.randn(P, H_kv, N_max, device="cuda", generator=g)
+    sc[0, 1] = torch.round(sc[0, 1] * 8) / 8
+    sc[1, 0] = -torch.rand(N_max, device="cuda", generator=g) - 1.0          # all negative
+    lens = torch.tensor([300001, 140000], dtype=torch.int32, device="cuda")
+    idx = torch.empty(P, H_kv, k, dtype=torch.int32, device="cuda")
+    keff = torch.empty(P, dtype=torch.int32, device="cuda")
+    mb.mage_topk(sc, lens, P, H_kv, N_max, k, idx, keff)
+    torch.cuda.synchronize()
+    from helpers import brute_force_topk
+    for p in range(P):
+        n = int(lens[p])
+        for h in range(H_kv):
+            ref = brute_force_topk(sc[p, h, :n].double().cpu().numpy(), k)
+            assert np.array_equal(idx[p, h].cpu().numpy(), ref), (p, h)
+
+
 def test_bad_indices_and_pages_are_flagged_not_dereferenced():
     """Host-made faults: an out-of-range index / page id sets a status bit and the row is skipped; nothing traps."""
     w = W.Workload("bad", H_q=8, H_kv=2, N=640, B=32, k=64, T=2, n_heavy=16, page_size=64, seed=2)
