@@ -269,3 +269,32 @@ def test_host_staged_blocks_match_the_resident_path(oracle_mod):
         for t in range(T):
             assert torch.equal(host_out[blk][t], expect[blk][t]), (blk, t)
     assert np.abs(expect[0][0].float().numpy() - res["outs"][0]).max() == 0.0
+
+
+def _random_shapes(n, seed):
+    rng = np.random.RandomState(seed)
+    shapes = []
+    for _ in range(n):
+        G, H_kv = int(rng.choice([1, 2, 4, 7, 8])), int(rng.choice([1, 2, 4]))
+        B = int(rng.choice([1, 4, 16, 32, 64]))
+        N = int(rng.choice([rng.randint(0, 200), rng.randint(200, 2000), rng.randint(2000, 9000)]))
+        k = int(rng.choice([16, 100, 512, 1024]))
+        P = int(rng.choice([1, 2, 3]))
+        paged = bool(rng.randint(0, 2))
+        ragged = bool(rng.randint(0, 2)) and N > 64
+        shapes.append((G * H_kv, H_kv, B, N, k, P, paged, ragged))
+    return shapes
+
+
+@pytest.mark.parametrize("shape", _random_shapes(12, seed=20260214), ids=lambda s: "x".join(str(int(v)) for v in s))
+def test_randomly_drawn_shapes(oracle_mod, shape):
+    """Shapes drawn at random (fixed seed): group size, KV heads, block size, prefix length, budget, batch, paged or not,
+    ragged or not -- every problem of each batch against the oracle."""
+    H_q, H_kv, B, N, k, P, paged, ragged = shape
+    w = W.Workload("drawn", H_q=H_q, H_kv=H_kv, N=N, B=B, k=k, T=2, P=P, n_heavy=min(32, N), seed=11,
+                   ragged_min=(N // 8 + 1) if ragged else 0, page_size=64 if paged else 0)
+    batch = W.make_batch(w, device="cuda")
+    res = H.run_gpu_block(batch, w, paged=paged)
+    assert res["status"] == 0
+    for p in range(P):
+        H.check_problem(oracle_mod, batch, res, w, p)
