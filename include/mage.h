@@ -24,6 +24,10 @@
  *     state between calls.  `stream` is a cudaStream_t passed as void*.
  *   - All calls only enqueue work on `stream` and return.  The return value
  *     covers host-detectable errors; nothing is launched when it is not MAGE_OK.
+ *     The tensor-core kernels are launched with the programmatic stream
+ *     serialization attribute and wait for their predecessor before they touch
+ *     global memory: ordering against other work in the stream is that of
+ *     ordinary stream order, and the calls may be captured into a CUDA graph.
  *   - Device-detectable problems (an index outside [0, N_p), a page id outside
  *     [0, num_pages), a bounded wait that expired) set bits in *dev_status
  *     (optional, may be NULL) and the offending access is skipped; a kernel
