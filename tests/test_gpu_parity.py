@@ -75,6 +75,23 @@ def test_strided_cache_view(oracle_mod, flags):
         H.check_problem(oracle_mod, batch, res, w, p)
 
 
+def test_padded_row_pitch(oracle_mod):
+    """Rows of 136 elements of which 128 are used: one row pitch for the whole cache (the reuse step's TMA row gather
+    and the dense tensor maps both take the pitch from the strides)."""
+    w = W.Workload("pitch", H_q=8, H_kv=2, N=1500, B=32, k=200, T=2, P=2, n_heavy=16, seed=10)
+    batch = W.make_batch(w, device="cuda")
+    def padded(x):
+        buf = torch.full(x.shape[:-1] + (136,), 7.0, dtype=x.dtype, device=x.device)
+        buf[..., :128] = x
+        return buf[..., :128]
+    b2 = dict(batch, kc=padded(batch["kc"]), vc=padded(batch["vc"]))
+    assert b2["kc"].stride(2) == 136 and not b2["kc"].is_contiguous()
+    res = H.run_gpu_block(b2, w)
+    assert res["status"] == 0
+    for p in range(w.P):
+        H.check_problem(oracle_mod, batch, res, w, p)
+
+
 @pytest.mark.parametrize("flags", IMPLS)
 def test_runs_are_bitwise_reproducible(flags):
     w = dataclasses.replace(W.CONFIGS["cfg1_small"], N=5000, T=2)
