@@ -318,7 +318,20 @@ def main():
         sp(); tk(); torch.cuda.synchronize()
         sp_cold, sp_warm, tk_ms = timed(sp, True), timed(sp, False), timed(tk, False)
         s1_ms = (sum(attn_ms) + sum(comb_ms) + sum(score_ms)) / len(attn_ms)
+
+        # Phase 1 as the paper arranges it (attention on the main stream; scores from Q and the cached keys plus top-k on the
+        # select stream; one join) against the fused form timed above (one call shares the rows' log-sum-exp).
+        def fused_phase1():
+            ba.exact_select(q_d[0], kb_d[0], vb_d[0], outs[0]); ba.select_async(); ba.join()
+
+        def two_stream_phase1():
+            ba.select_scores_async(q_d[0]); ba.exact_attn(q_d[0], kb_d[0], vb_d[0], outs[0]); ba.join()
+
+        sel_alone = lambda: mb.mage_select_scores(kv, q_d[0], ba.sm_scale, ba.scores, ba._select_workspace, ba.status)
+        two_stream_phase1(); torch.cuda.synchronize()
+        p1_fused, p1_two, sel_ms = timed(fused_phase1, False, 5), timed(two_stream_phase1, False, 5), timed(sel_alone, False, 5)
         stages = {
+            "phase1_fused_ms": p1_fused, "phase1_two_stream_ms": p1_two, "select_scores_ms_alone": sel_ms,
             "exact_select_ms": s1_ms, "attn_kernel_ms": sum(attn_ms) / len(attn_ms), "combine_kernel_ms": sum(comb_ms) / len(comb_ms),
             "score_kernel_ms": sum(score_ms) / len(score_ms),
             "exact_select_gbs": sf["s1_bytes"] / s1_ms / 1e6, "exact_select_frac_of_8tbs": sf["s1_bytes"] / s1_ms / 1e6 / 8000.0,

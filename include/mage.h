@@ -176,6 +176,35 @@ mage_status mage_append_block(const mage_kv_t *kv, const void *k_blk, const void
                               uint32_t *dev_status, void *stream);
 
 /*
+ * The main stream's half of Step 1 on its own (Algorithm 1, main stream:
+ * "Attn(Q, K, V, C)"): exact attention of the block over the prefix cache and its
+ * own keys, no block scores.  Arguments, layouts and errors as mage_exact_select
+ * (which is this call followed by the score pass, sharing the rows' log-sum-exp).
+ */
+mage_status mage_exact_attn(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk, float sm_scale,
+                            void *out, void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream);
+
+/*
+ * The select stream's computation on its own (Algorithm 1, select stream:
+ * "A = softmax(Q K^T / sqrt d)" over the prefix cache, then Eq. 4's mean over the
+ * block's G*B rows), without the attention output: block scores from the queries
+ * and the cached keys alone.  For callers that run the selection beside the main
+ * stream's attention as the paper does, rather than reuse mage_exact_select's pass.
+ * Work: one pass over K for the rows' log-sum-exp (no V, no block keys), one pass
+ * for the scores.  The scores are bit-identical to mage_exact_select's.
+ *
+ *   q          [P][H_q][B][d] bf16, device.
+ *   scores     [P][H_kv][N_max] fp32, device, written for positions < N_p; may be
+ *              NULL only when N_max == 0.
+ *   workspace  device, 256-byte aligned, at least mage_workspace_bytes(kv, k_max)
+ *              for any k_max >= 1; it must not be the workspace of a call that may
+ *              run at the same time on another stream.
+ * Errors: as mage_exact_select.
+ */
+mage_status mage_select_scores(const mage_kv_t *kv, const void *q, float sm_scale, float *scores, void *workspace,
+                               size_t workspace_bytes, uint32_t *dev_status, void *stream);
+
+/*
  * Step 1 of a block for callers that cannot hand over a workspace (the paper has no counterpart; this is a
  * packaging variant of mage_exact_select, same arithmetic, same kernels).
  *

@@ -38,7 +38,7 @@ class mage_kv_t(ctypes.Structure):
     ]
 
 
-EXPORTS = ("mage_append_block", "mage_workspace_bytes", "mage_exact_select", "mage_exact_select_events", "mage_exact_select_static", "mage_topk", "mage_sparse_block_attn",
+EXPORTS = ("mage_append_block", "mage_workspace_bytes", "mage_exact_select", "mage_exact_select_events", "mage_exact_select_static", "mage_exact_attn", "mage_select_scores", "mage_topk", "mage_sparse_block_attn",
            "mage_status_string", "mage_launch_count")
 
 
@@ -59,6 +59,10 @@ def load():
     lib.mage_exact_select_events.argtypes = lib.mage_exact_select.argtypes + [ctypes.POINTER(ctypes.c_void_p)]
     lib.mage_exact_select_static.restype = ctypes.c_int
     lib.mage_exact_select_static.argtypes = [ctypes.POINTER(mage_kv_t), vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
+    lib.mage_exact_attn.restype = ctypes.c_int
+    lib.mage_exact_attn.argtypes = [ctypes.POINTER(mage_kv_t), vp, vp, vp, ctypes.c_float, vp, vp, ctypes.c_size_t, vp, vp]
+    lib.mage_select_scores.restype = ctypes.c_int
+    lib.mage_select_scores.argtypes = [ctypes.POINTER(mage_kv_t), vp, ctypes.c_float, vp, vp, ctypes.c_size_t, vp, vp]
     lib.mage_topk.restype = ctypes.c_int
     lib.mage_topk.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, ctypes.c_size_t, vp]
     lib.mage_sparse_block_attn.restype = ctypes.c_int
@@ -157,6 +161,24 @@ def mage_exact_select(kv: KVCache, q, k_blk, v_blk, sm_scale: float, out, scores
         rc = load().mage_exact_select_events(*args, handles)
     if rc != MAGE_OK:
         raise MageError(rc, "mage_exact_select")
+
+
+def mage_exact_attn(kv: KVCache, q, k_blk, v_blk, sm_scale: float, out, workspace, dev_status=None, stream=None):
+    """Exact attention of the block without the score pass (the main stream's half of Step 1; see mage.h)."""
+    ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    rc = load().mage_exact_attn(ctypes.byref(kv.c), _ptr(q), _ptr(k_blk), _ptr(v_blk), float(sm_scale), _ptr(out), _ptr(workspace),
+                                ws_bytes, _ptr(dev_status), _stream(stream))
+    if rc != MAGE_OK:
+        raise MageError(rc, "mage_exact_attn")
+
+
+def mage_select_scores(kv: KVCache, q, sm_scale: float, scores, workspace, dev_status=None, stream=None):
+    """Block scores from the queries and the cached keys alone (the select stream's own computation; see mage.h)."""
+    ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    rc = load().mage_select_scores(ctypes.byref(kv.c), _ptr(q), float(sm_scale), _ptr(scores), _ptr(workspace), ws_bytes,
+                                   _ptr(dev_status), _stream(stream))
+    if rc != MAGE_OK:
+        raise MageError(rc, "mage_select_scores")
 
 
 STATIC_SCRATCH_BYTES = 32 << 20

@@ -150,22 +150,31 @@ static mage_status opt_in_smem(K kernel, size_t bytes) { return opt_in_smem_impl
 static mage_status exact_select_simt(const mage_kv_t *kv, const KvView &view, const Plan &plan, const __nv_bfloat16 *q,
                                      const __nv_bfloat16 *k_blk, const __nv_bfloat16 *v_blk, float sm_scale,
                                      __nv_bfloat16 *out, float *scores, float *ws, unsigned *dev_status, cudaStream_t st,
-                                     cudaEvent_t *ev) {
+                                     cudaEvent_t *ev, bool scores_only = false) {
+    // scores_only: the select stream's own computation (Algorithm 1: A = softmax(Q K^T / sqrt d) over the prefix, then
+    // the mean over the block's rows) without the attention output: pass A keeps only the rows' maxima and sums (no V,
+    // no P V, no block keys), the merge emits only the log-sum-exp, pass B is unchanged.  k_blk, v_blk, out are unused.
     using namespace simt;
     const float scale_log2 = sm_scale * kLog2e;
     auto kern = attn_kernel<Mode::kExactPartial>;
     if (opt_in_smem(kern, kSmemBytes) != MAGE_OK || opt_in_smem(simt::score_kernel, kSmemBytes) != MAGE_OK) return MAGE_ERR_CUDA;
     const int row_tiles = (view.M + kRows - 1) / kRows;
-    dim3 grid(row_tiles, plan.n_chunks + 1, kv->P * kv->H_kv);
+    dim3 grid(row_tiles, plan.n_chunks + (scores_only ? 0 : 1), kv->P * kv->H_kv);
     if (ev) cudaEventRecord(ev[0], st);
     bool tc_attn_done = false;
     if (tc::eligible(kv)) {
         tc::AttnMaps maps;
         auto kern_tc = tc::attn_kernel<false>;
-        if (tc::make_group_rows_map(&maps.q, q, (long long)kv->P * kv->H_kv, kv->H_q / kv->H_kv * kv->B) && tc::make_cache_map(&maps.k, kv, kv->k_cache) &&
-            tc::make_cache_map(&maps.v, kv, kv->v_cache) && tc::make_rows_map(&maps.kb, k_blk, (long long)kv->P * kv->H_kv * kv->B) &&
-            tc::make_rows_map(&maps.vb, v_blk, (long long)kv->P * kv->H_kv * kv->B) && opt_in_smem(kern_tc, tc::kAttnSmemBytesDense) == MAGE_OK) {
-            dim3 tgrid(plan.n_chunks + 1, (view.M + 255) / 256, kv->P * kv->H_kv);
+        bool maps_ok = tc::make_group_rows_map(&maps.q, q, (long long)kv->P * kv->H_kv, kv->H_q / kv->H_kv * kv->B) && tc::make_cache_map(&maps.k, kv, kv->k_cache);
+        if (maps_ok && scores_only) {
+            maps.v = maps.kb = maps.vb = maps.k;          // never used in this mode
+            maps.lse_only = 1;
+        } else if (maps_ok) {
+            maps_ok = tc::make_cache_map(&maps.v, kv, kv->v_cache) && tc::make_rows_map(&maps.kb, k_blk, (long long)kv->P * kv->H_kv * kv->B) &&
+                      tc::make_rows_map(&maps.vb, v_blk, (long long)kv->P * kv->H_kv * kv->B);
+        }
+        if (maps_ok && plan.n_chunks + (scores_only ? 0 : 1) > 0 && opt_in_smem(kern_tc, tc::kAttnSmemBytesDense) == MAGE_OK) {
+            dim3 tgrid(plan.n_chunks + (scores_only ? 0 : 1), (view.M + 255) / 256, kv->P * kv->H_kv);
             launch_pdl(kern_tc, tgrid, dim3(320), tc::kAttnSmemBytesDense, st, maps, view, plan, k_blk, v_blk, (const int *)nullptr, (const int *)nullptr, 0, scale_log2, ws,
                        (__nv_bfloat16 *)nullptr, dev_status);
             if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
@@ -178,9 +187,10 @@ static mage_status exact_select_simt(const mage_kv_t *kv, const KvView &view, co
     }
     if (ev) cudaEventRecord(ev[1], st);
     const int rows_total = kv->P * kv->H_kv * view.M;
-    launch_pdl(combine_kernel, dim3((rows_total + 3) / 4), dim3(128), 0, st, view, plan, ws, out);
+    launch_pdl(combine_kernel, dim3((rows_total + 3) / 4), dim3(128), 0, st, view, plan, ws, out, (int)scores_only);
     if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
     if (ev) cudaEventRecord(ev[2], st);
+    if (!scores) return MAGE_OK;                          // attention only (the main stream of the two-stream arrangement)
     bool tc_score_done = false;
     if (tc::eligible(kv)) {
         CUtensorMap map_q, map_k;
@@ -285,6 +295,34 @@ mage_status mage_exact_select(const mage_kv_t *kv, const void *q, const void *k_
                               void *stream) {
     return mage_exact_select_events(kv, q, k_blk, v_blk, sm_scale, out, scores, workspace, workspace_bytes, dev_status,
                                     stream, nullptr);
+}
+
+mage_status mage_exact_attn(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk, float sm_scale,
+                            void *out, void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream) {
+    mage_status why = MAGE_OK;
+    if (!valid_kv(kv, &why)) return why;
+    if (!q || !k_blk || !v_blk || !out || !workspace) return MAGE_ERR_INVALID_ARG;
+    if (!(sm_scale > 0.f) || (reinterpret_cast<uintptr_t>(workspace) & 255)) return MAGE_ERR_INVALID_ARG;
+    const Plan plan = make_plan(kv);
+    if (workspace_bytes < plan.exact_bytes) return MAGE_ERR_WORKSPACE;
+    const KvView view = make_view(kv);
+    return exact_select_simt(kv, view, plan, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_blk),
+                             static_cast<const __nv_bfloat16 *>(v_blk), sm_scale, static_cast<__nv_bfloat16 *>(out), nullptr,
+                             static_cast<float *>(workspace), dev_status, static_cast<cudaStream_t>(stream), nullptr);
+}
+
+mage_status mage_select_scores(const mage_kv_t *kv, const void *q, float sm_scale, float *scores, void *workspace,
+                               size_t workspace_bytes, uint32_t *dev_status, void *stream) {
+    mage_status why = MAGE_OK;
+    if (!valid_kv(kv, &why)) return why;
+    if (!q || !workspace || (kv->N_max > 0 && !scores)) return MAGE_ERR_INVALID_ARG;
+    if (!(sm_scale > 0.f) || (reinterpret_cast<uintptr_t>(workspace) & 255)) return MAGE_ERR_INVALID_ARG;
+    const Plan plan = make_plan(kv);
+    if (workspace_bytes < plan.exact_bytes) return MAGE_ERR_WORKSPACE;
+    if (kv->N_max == 0) return MAGE_OK;                   // no prefix: no score to write
+    const KvView view = make_view(kv);
+    return exact_select_simt(kv, view, plan, static_cast<const __nv_bfloat16 *>(q), nullptr, nullptr, sm_scale, nullptr, scores,
+                             static_cast<float *>(workspace), dev_status, static_cast<cudaStream_t>(stream), nullptr, true);
 }
 
 mage_status mage_topk(const float *scores, const int32_t *seq_lens, int32_t P, int32_t H_kv, int32_t N_max, int32_t k,

@@ -258,7 +258,7 @@ __global__ void __launch_bounds__(kThreads) score_kernel(KvView kv, Plan plan, c
 //  - log-sum-exp over the prefix chunks only -> neg_lse (log2 domain), used by the score kernels;
 //  - prefix chunks + the block's own keys -> normalised bf16 output.
 __global__ void __launch_bounds__(128) combine_kernel(KvView kv, Plan plan, float *__restrict__ ws,
-                                                      __nv_bfloat16 *__restrict__ out) {
+                                                      __nv_bfloat16 *__restrict__ out, int lse_only) {
     // may have been launched while the attention kernel was still running (programmatic dependent launch): wait for it,
     // then let the score kernel's CTAs be scheduled
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -297,6 +297,7 @@ __global__ void __launch_bounds__(128) combine_kernel(KvView kv, Plan plan, floa
 #pragma unroll
     for (int w = 16; w; w >>= 1) l_pre += __shfl_xor_sync(0xffffffffu, l_pre, w);
     if (lane == 0) ws[plan.off_neg_lse + (size_t)z * plan.Mw + r] = nc > 0 ? -(m_pre + log2f(l_pre)) : 0.f;
+    if (lse_only) return;                                 // the select stream's own pass: no block chunk, no output
     const float *eb = ml + ((item0 + plan.n_chunks) * plan.Mw + r) * 2;
     const float m_blk = eb[0], l_blk = eb[1];
     const float m_all = fmaxf(m_pre, m_blk);

@@ -316,9 +316,10 @@ constexpr size_t kAttnSmemBytesSparse = 1024 + kAttnQBytes + kAttnSlotsSparse * 
 constexpr float kRescaleThreshold = 8.f;               // log2 units
 
 // gather_rows > 0 (reuse step only): k, v, kb, vb are flat row lists (pitch gather_pitch elements) with 64 x 1 boxes.
+// lse_only (exact pass only): the select stream's own pass -- row maxima and sums over the prefix, no V, no P V, no O.
 struct AttnMaps {
     CUtensorMap q, k, v, kb, vb;
-    int gather_rows = 0, gather_blk_rows = 0, gather_pitch = 0;
+    int gather_rows = 0, gather_blk_rows = 0, gather_pitch = 0, lse_only = 0;
 };
 
 template <bool SPARSE>
@@ -428,6 +429,11 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 for (int L = 0; L < 2 * n_tiles; ++L) {
                     const int i = L >> 1, is_v = L & 1, slot = slot_of(L);
                     if (!mbar_wait(bar(EMPTY + slot), par_of(L) ^ 1, abort_s, status)) break;
+                    if (maps.lse_only && is_v) {               // no values in this mode: the slot's phase is completed empty-handed
+                        mbar_arrive(bar(FULL + slot));
+                        issued = L + 1;
+                        continue;
+                    }
                     mbar_arrive_expect_tx(bar(FULL + slot), kTileBytes);
                     const uint32_t dst = smem_u32(kv_s + slot * kTileBytes);
                     for (int kh = 0; kh < 2; ++kh) {
@@ -578,6 +584,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             };
             // half 0: keys 0-63 of the tile, half 1: keys 64-127; 16 keys per step = 16 rows of 128 bytes in each d-half
             auto pv = [&](int slot, int reg, int half, uint32_t acc) {
+                if (maps.lse_only) return;
                 const uint32_t b0 = v_lo + (uint32_t)slot * kTileU;
 #pragma unroll
                 for (int ks = half * 4; ks < half * 4 + 4; ++ks)
@@ -967,7 +974,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 };
                 auto store_partial = [&](float *po_row0, float *pml_row) {                  // unnormalised O, then (m, l)
 #pragma unroll 1
-                    for (int c0 = 0; c0 < kD; c0 += 64) {
+                    for (int c0 = 0; c0 < (maps.lse_only ? 0 : kD); c0 += 64) {
 #pragma unroll 1
                         for (int c1 = 0; c1 < 64; c1 += 32) {
                             uint32_t r[32];

@@ -42,6 +42,28 @@ class BlockAttention:
                              events)
         return out
 
+    def exact_attn(self, q, k_blk, v_blk, out=None, stream=None):
+        """Step 1's attention alone on ``stream`` (default: current); pair it with ``select_scores_async``."""
+        out = self.out if out is None else out
+        mb.mage_exact_attn(self.kv, q, k_blk, v_blk, self.sm_scale, out, self.workspace, self.status, stream)
+        return out
+
+    def select_scores_async(self, q, workspace: Optional[torch.Tensor] = None, main_stream=None):
+        """The paper's two-stream Phase 1: block scores and top-k on the select stream from the queries alone, beside
+        whatever the main stream does (its attention, then the FFN).  Uses a workspace of its own (allocated on first use),
+        since the main stream's Step 1 may be using ``self.workspace`` at the same time.  Follow with ``join()``."""
+        main = torch.cuda.current_stream() if main_stream is None else main_stream
+        if workspace is None:
+            if getattr(self, "_select_workspace", None) is None:
+                self._select_workspace = self.kv.new_workspace(self.k)
+            workspace = self._select_workspace
+        self._scores_ready.record(main)                   # q is ready on the main stream
+        self.select_stream.wait_event(self._scores_ready)
+        mb.mage_select_scores(self.kv, q, self.sm_scale, self.scores, workspace, self.status, self.select_stream)
+        mb.mage_topk(self.scores, self.kv.seq_lens, self.kv.P, self.kv.H_kv, max(self.kv.N_max, 0), self.k, self.indices,
+                     self.k_eff, stream=self.select_stream)
+        self._indices_ready.record(self.select_stream)
+
     def select_async(self, main_stream=None):
         """Top-k on the select stream, ordered after the scores written on ``main_stream``; does not block it."""
         main = torch.cuda.current_stream() if main_stream is None else main_stream

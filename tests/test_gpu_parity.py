@@ -315,3 +315,36 @@ def test_randomly_drawn_shapes(oracle_mod, shape):
     assert res["status"] == 0
     for p in range(P):
         H.check_problem(oracle_mod, batch, res, w, p)
+
+
+@pytest.mark.parametrize("flags", IMPLS)
+@pytest.mark.parametrize("shape", [(8, 2, 32, 5000, 2), (28, 4, 32, 9000, 3), (14, 2, 64, 700, 1)], ids=lambda s: "x".join(map(str, s)))
+def test_select_stream_scores_alone(oracle_mod, flags, shape):
+    """mage_select_scores (Algorithm 1's select stream on its own: scores from Q and the cached keys, no attention output)
+    gives the scores of mage_exact_select bit for bit, with ragged lengths and pages, and the two-stream pipeline built on
+    it selects the same sets."""
+    H_q, H_kv, B, N, P = shape
+    w = W.Workload("select_only", H_q=H_q, H_kv=H_kv, N=N, B=B, k=128, T=2, P=P, n_heavy=32, seed=21,
+                   ragged_min=N // 4 if P > 1 else 0, page_size=64 if P == 3 else 0)
+    batch = W.make_batch(w, device="cuda")
+    res = H.run_gpu_block(batch, w, paged=(P == 3), flags=flags)
+    ba = res["ba"]
+    fused_scores, fused_idx = ba.scores.clone(), ba.indices.clone()
+    ba.scores.fill_(-1.0)
+    ws2 = ba.kv.new_workspace(w.k)
+    mb.mage_select_scores(ba.kv, batch["q"][0], ba.sm_scale, ba.scores, ws2, ba.status)
+    torch.cuda.synchronize()
+    assert int(ba.status.item()) == 0
+    lens = batch["seq_lens"].tolist()
+    for p in range(P):
+        assert torch.equal(ba.scores[p, :, :lens[p]], fused_scores[p, :, :lens[p]]), p
+        assert (ba.scores[p, :, lens[p]:] == -1.0).all()
+    # the paper's arrangement: attention on the main stream, scores + top-k on the select stream, one join
+    ba.indices.fill_(-7)
+    out = torch.empty_like(ba.out)
+    ba.select_scores_async(batch["q"][0])
+    ba.exact_attn(batch["q"][0], batch["kb"][0], batch["vb"][0], out)
+    ba.join()
+    torch.cuda.synchronize()
+    assert torch.equal(ba.indices, fused_idx)
+    assert np.array_equal(out.float().cpu().numpy(), res["outs"][0])
