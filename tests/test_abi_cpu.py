@@ -62,6 +62,26 @@ def test_workspace_bytes_is_pure_host_arithmetic(lib):
     assert 0 < lib.mage_workspace_bytes(ctypes.byref(big), 512) < (1 << 30)
 
 
+def test_workspace_plan_over_a_range_of_shapes(lib):
+    """The chunk count behind the workspace size comes from a cost search; whatever it picks, the size stays bounded
+    (at most 148 partial results per head plus the split region), grows with the budget, and one Qwen-shaped layer at
+    32K fits the 32 MiB of the no-allocation entry point."""
+    from paper_2602_14209_b200 import binding
+    per_item = 256 * (128 + 2) * 4                       # one partial result of a 224-row head: O and (m, l), fp32
+    for P in (1, 3, 28, 200):
+        for N in (0, 100, 2048, 32768, 131072, 1000000):
+            for page in (0, 64):
+                c = _kv(P=P, H_q=28, H_kv=4, N_max=N, stride_h=max(N, 1) * 128, stride_p=4 * max(N, 1) * 128, page_size=page)
+                if page:
+                    c.block_table, c.max_pages, c.num_pages = 4096, (N + page - 1) // page, max(1, P * ((N + page - 1) // page))
+                small, large = lib.mage_workspace_bytes(ctypes.byref(c), 64), lib.mage_workspace_bytes(ctypes.byref(c), 2048)
+                heads = P * 4
+                assert 0 < small <= large, (P, N, page)
+                assert small <= heads * (149 + 33) * per_item + (1 << 20), (P, N, page, small)
+    layer = _kv(P=1, H_q=28, H_kv=4, N_max=32768, stride_h=32768 * 128, stride_p=4 * 32768 * 128)
+    assert lib.mage_workspace_bytes(ctypes.byref(layer), 512) <= binding.STATIC_SCRATCH_BYTES + (8 << 20)
+
+
 @pytest.mark.parametrize("over,code", [
     (dict(d=64), -2), (dict(B=65), -2), (dict(B=0), -1), (dict(H_q=9), -1), (dict(P=0), -1),
     (dict(stride_n=100), -1), (dict(stride_h=12), -1), (dict(k_cache=0), -1), (dict(page_size=-1), -1),
