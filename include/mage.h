@@ -60,7 +60,14 @@ typedef enum {
 #define MAGE_DEV_CACHE_FULL 8u  /* mage_append_block: no room left for the block: nothing appended for that problem */
 
 /* mage_kv_t.flags */
-#define MAGE_FLAG_SIMT_KERNELS 1  /* use the portable CUDA-core kernels for every stage (slow; for cross-checks) */
+#define MAGE_FLAG_SIMT_KERNELS 1  /* use the portable CUDA-core kernels for every stage (about 25x slower; for cross-checks
+                                     and for layouts the tensor-core kernels do not take).  The library never switches to
+                                     them by itself: without this flag, a description that the tensor-core kernels cannot
+                                     take is refused with MAGE_ERR_UNSUPPORTED and nothing is launched.  That concerns:
+                                     page sizes that are not multiples of 64, k_cache / v_cache (or, in the reuse step,
+                                     k_blk / v_blk) not 16-byte aligned, strides or extents that a TMA tensor map cannot
+                                     express, and, in the reuse step on a cache that is not one list of rows with a single
+                                     pitch, a cache of more than 2^34 elements. */
 
 /*
  * Prefix KV cache "C" of Algorithm 1 for a batch of P problems, read-only.
@@ -72,12 +79,12 @@ typedef enum {
  * logical position j of problem p lives in pool page block_table[p*max_pages + j/page_size],
  * row j % page_size.  Strides are ignored.
  * seq_lens[p] = N_p <= N_max is the prefix length of problem p (NULL: every N_p = N_max).
- * N_p = 0 is legal.  Cache rows at positions >= N_p are never used as data.
+ * N_p = 0 is legal.  Cache rows at positions >= N_p are never used as data.  P * H_kv <= 65535.
  */
 typedef struct mage_kv {
     int32_t P, H_q, H_kv, d;      /* d must be 128; H_q % H_kv == 0                    */
     int32_t B;                    /* 1..64 block tokens                                */
-    int32_t page_size;            /* 0 = contiguous, else tokens per page (power of two >= 16) */
+    int32_t page_size;            /* 0 = contiguous, else tokens per page (power of two >= 16; see MAGE_FLAG_SIMT_KERNELS) */
     const void *k_cache, *v_cache;
     int64_t stride_p, stride_h, stride_n;
     const int32_t *block_table;   /* device [P][max_pages], paged only                 */

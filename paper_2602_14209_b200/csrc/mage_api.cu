@@ -32,7 +32,7 @@ static bool valid_kv(const mage_kv_t *kv, mage_status *why) {
         if (kv->N_max > 0 && (!kv->block_table || kv->num_pages < 1)) return fail(MAGE_ERR_INVALID_ARG);
         if ((int64_t)kv->max_pages * kv->page_size < kv->N_max) return fail(MAGE_ERR_INVALID_ARG);
     }
-    if ((int64_t)kv->P * kv->H_kv > 65535 * 16) return fail(MAGE_ERR_UNSUPPORTED);
+    if ((int64_t)kv->P * kv->H_kv > 65535) return fail(MAGE_ERR_UNSUPPORTED);      // (problem, KV head) pairs are one grid dimension
     return true;
 }
 
@@ -147,120 +147,146 @@ static mage_status opt_in_smem_impl(const void *kernel, size_t bytes) {
 template <typename K>
 static mage_status opt_in_smem(K kernel, size_t bytes) { return opt_in_smem_impl(reinterpret_cast<const void *>(kernel), bytes); }
 
-static mage_status exact_select_simt(const mage_kv_t *kv, const KvView &view, const Plan &plan, const __nv_bfloat16 *q,
-                                     const __nv_bfloat16 *k_blk, const __nv_bfloat16 *v_blk, float sm_scale,
-                                     __nv_bfloat16 *out, float *scores, float *ws, unsigned *dev_status, cudaStream_t st,
-                                     cudaEvent_t *ev, bool scores_only = false) {
-    // scores_only: the select stream's own computation (Algorithm 1: A = softmax(Q K^T / sqrt d) over the prefix, then
-    // the mean over the block's rows) without the attention output: pass A keeps only the rows' maxima and sums (no V,
-    // no P V, no block keys), the merge emits only the log-sum-exp, pass B is unchanged.  k_blk, v_blk, out are unused.
-    using namespace simt;
+// Why the tensor-core kernels cannot take this description, or MAGE_OK.  There is one production path; the portable
+// CUDA-core kernels run only when the caller asks for them with MAGE_FLAG_SIMT_KERNELS, never as a silent substitute.
+static mage_status tc_supported(const mage_kv_t *kv) {
+    if (kv->page_size != 0 && kv->page_size % 64 != 0) return MAGE_ERR_UNSUPPORTED;        // a 64-key TMA box must lie inside one page
+    if (kv->N_max > 0 && ((reinterpret_cast<uintptr_t>(kv->k_cache) | reinterpret_cast<uintptr_t>(kv->v_cache)) & 15)) return MAGE_ERR_UNSUPPORTED;
+    if (tc::encode_fn() == nullptr) return MAGE_ERR_CUDA;
+    return MAGE_OK;
+}
+
+// Step 1 (Algorithm 1, Phase 1): the exact pass over prefix + block keys, the merge of its per-chunk partial results and
+// the block-score pass.  scores_only: the select stream's own computation (Algorithm 1: A = softmax(Q K^T / sqrt d) over
+// the prefix, then the mean over the block's rows) without the attention output: pass A keeps only the rows' maxima and
+// sums (no V, no P V, no block keys), the merge emits only the log-sum-exp, pass B is unchanged; k_blk, v_blk, out unused.
+static mage_status launch_exact_select(const mage_kv_t *kv, const KvView &view, const Plan &plan, const __nv_bfloat16 *q,
+                                       const __nv_bfloat16 *k_blk, const __nv_bfloat16 *v_blk, float sm_scale,
+                                       __nv_bfloat16 *out, float *scores, float *ws, unsigned *dev_status, cudaStream_t st,
+                                       cudaEvent_t *ev, bool scores_only = false) {
     const float scale_log2 = sm_scale * kLog2e;
-    auto kern = attn_kernel<Mode::kExactPartial>;
-    if (opt_in_smem(kern, kSmemBytes) != MAGE_OK || opt_in_smem(simt::score_kernel, kSmemBytes) != MAGE_OK) return MAGE_ERR_CUDA;
-    const int row_tiles = (view.M + kRows - 1) / kRows;
-    dim3 grid(row_tiles, plan.n_chunks + (scores_only ? 0 : 1), kv->P * kv->H_kv);
-    if (ev) cudaEventRecord(ev[0], st);
-    bool tc_attn_done = false;
-    if (tc::eligible(kv)) {
-        tc::AttnMaps maps;
-        auto kern_tc = tc::attn_kernel<false>;
-        bool maps_ok = tc::make_group_rows_map(&maps.q, q, (long long)kv->P * kv->H_kv, kv->H_q / kv->H_kv * kv->B) && tc::make_cache_map(&maps.k, kv, kv->k_cache);
-        if (maps_ok && scores_only) {
-            maps.v = maps.kb = maps.vb = maps.k;          // never used in this mode
-            maps.lse_only = 1;
-        } else if (maps_ok) {
-            maps_ok = tc::make_cache_map(&maps.v, kv, kv->v_cache) && tc::make_rows_map(&maps.kb, k_blk, (long long)kv->P * kv->H_kv * kv->B) &&
-                      tc::make_rows_map(&maps.vb, v_blk, (long long)kv->P * kv->H_kv * kv->B);
-        }
-        if (maps_ok && plan.n_chunks + (scores_only ? 0 : 1) > 0 && opt_in_smem(kern_tc, tc::kAttnSmemBytesDense) == MAGE_OK) {
-            dim3 tgrid(plan.n_chunks + (scores_only ? 0 : 1), (view.M + 255) / 256, kv->P * kv->H_kv);
-            launch_pdl(kern_tc, tgrid, dim3(320), tc::kAttnSmemBytesDense, st, maps, view, plan, k_blk, v_blk, (const int *)nullptr, (const int *)nullptr, 0, scale_log2, ws,
-                       (__nv_bfloat16 *)nullptr, dev_status);
+    const int heads = kv->P * kv->H_kv, rows_total = heads * view.M;
+    const int n_items = plan.n_chunks + (scores_only ? 0 : 1);
+    if (kv->flags & MAGE_FLAG_SIMT_KERNELS) {
+        using namespace simt;
+        auto kern = attn_kernel<Mode::kExactPartial>;
+        if (opt_in_smem(kern, kSmemBytes) != MAGE_OK || opt_in_smem(simt::score_kernel, kSmemBytes) != MAGE_OK) return MAGE_ERR_CUDA;
+        if (ev) cudaEventRecord(ev[0], st);
+        if (n_items > 0) {
+            kern<<<dim3((view.M + kRows - 1) / kRows, n_items, heads), kThreads, kSmemBytes, st>>>(view, plan, q, k_blk, v_blk, nullptr, nullptr, 0, scale_log2, ws, nullptr, dev_status);
             if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
-            tc_attn_done = true;
         }
+        if (ev) cudaEventRecord(ev[1], st);
+        launch_pdl(combine_kernel, dim3((rows_total + 3) / 4), dim3(128), 0, st, view, plan, ws, out, (int)scores_only);
+        if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+        if (ev) cudaEventRecord(ev[2], st);
+        if (scores && kv->N_max > 0) {
+            simt::score_kernel<<<dim3((kv->N_max + kKeys - 1) / kKeys, 1, heads), kThreads, kSmemBytes, st>>>(view, plan, q, scale_log2, ws, scores, dev_status);
+            if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+        }
+        if (ev) cudaEventRecord(ev[3], st);
+        return MAGE_OK;
     }
-    if (!tc_attn_done) {
-        kern<<<grid, kThreads, kSmemBytes, st>>>(view, plan, q, k_blk, v_blk, nullptr, nullptr, 0, scale_log2, ws, nullptr, dev_status);
+    const mage_status sup = tc_supported(kv);
+    if (sup != MAGE_OK) return sup;
+    // every tensor map is encoded before the first launch: a description that cannot be encoded launches nothing
+    tc::AttnMaps maps;
+    CUtensorMap map_q_rows, map_k_score;
+    auto kern_tc = tc::attn_kernel<false>;
+    bool maps_ok = tc::make_group_rows_map(&maps.q, q, heads, view.M);
+    if (maps_ok && kv->N_max > 0) maps_ok = tc::make_cache_map(&maps.k, kv, kv->k_cache);
+    else maps.k = maps.q;                                  // no prefix: never used
+    if (maps_ok && scores_only) {
+        maps.v = maps.kb = maps.vb = maps.k;              // never used in this mode
+        maps.lse_only = 1;
+    } else if (maps_ok) {
+        maps_ok = tc::make_rows_map(&maps.kb, k_blk, (long long)heads * kv->B) && tc::make_rows_map(&maps.vb, v_blk, (long long)heads * kv->B);
+        if (maps_ok && kv->N_max > 0) maps_ok = tc::make_cache_map(&maps.v, kv, kv->v_cache);
+        else maps.v = maps.q;
+    }
+    const bool want_scores = scores && kv->N_max > 0;
+    if (maps_ok && want_scores) maps_ok = tc::make_rows_map(&map_q_rows, q, (long long)kv->P * kv->H_q * kv->B) && tc::make_cache_map(&map_k_score, kv, kv->k_cache);
+    if (!maps_ok) return MAGE_ERR_UNSUPPORTED;
+    if (opt_in_smem(kern_tc, tc::kAttnSmemBytesDense) != MAGE_OK || opt_in_smem(tc::score_kernel, tc::kScoreSmemBytes) != MAGE_OK) return MAGE_ERR_CUDA;
+    if (ev) cudaEventRecord(ev[0], st);
+    if (n_items > 0) {
+        launch_pdl(kern_tc, dim3(n_items, (view.M + 255) / 256, heads), dim3(320), tc::kAttnSmemBytesDense, st, maps, view, plan, k_blk, v_blk, (const int *)nullptr,
+                   (const int *)nullptr, 0, scale_log2, ws, (__nv_bfloat16 *)nullptr, dev_status);
         if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
     }
     if (ev) cudaEventRecord(ev[1], st);
-    const int rows_total = kv->P * kv->H_kv * view.M;
     launch_pdl(combine_kernel, dim3((rows_total + 3) / 4), dim3(128), 0, st, view, plan, ws, out, (int)scores_only);
     if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
     if (ev) cudaEventRecord(ev[2], st);
-    if (!scores) return MAGE_OK;                          // attention only (the main stream of the two-stream arrangement)
-    bool tc_score_done = false;
-    if (tc::eligible(kv)) {
-        CUtensorMap map_q, map_k;
-        if (tc::make_rows_map(&map_q, q, (long long)kv->P * kv->H_q * kv->B) && tc::make_cache_map(&map_k, kv, kv->k_cache) &&
-            opt_in_smem(tc::score_kernel, tc::kScoreSmemBytes) == MAGE_OK) {
-            const int tpc = tc::tiles_per_cta_for((long long)kv->P * kv->H_kv, kv->N_max, kv->page_size != 0);
-            const int tiles_head = (kv->N_max + tc::kTile - 1) / tc::kTile;
-            dim3 sgrid((tiles_head + tpc - 1) / tpc, kv->P * kv->H_kv, 1);
-            for (int r0 = 0; r0 < view.M; r0 += 256) {
-                launch_pdl(tc::score_kernel, sgrid, dim3(tc::kScoreThreads), tc::kScoreSmemBytes, st, map_q, map_k, view, plan, r0, std::min(256, view.M - r0),
-                           tpc, scale_log2, (const float *)ws, scores, (int)(r0 > 0), dev_status);
-                if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
-            }
-            tc_score_done = true;
+    if (want_scores) {
+        const int tpc = tc::tiles_per_cta_for(heads, kv->N_max, kv->page_size != 0);
+        const int tiles_head = (kv->N_max + tc::kTile - 1) / tc::kTile;
+        dim3 sgrid((tiles_head + tpc - 1) / tpc, heads, 1);
+        for (int r0 = 0; r0 < view.M; r0 += 256) {
+            launch_pdl(tc::score_kernel, sgrid, dim3(tc::kScoreThreads), tc::kScoreSmemBytes, st, map_q_rows, map_k_score, view, plan, r0, std::min(256, view.M - r0),
+                       tpc, scale_log2, (const float *)ws, scores, (int)(r0 > 0), dev_status);
+            if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
         }
-    }
-    if (!tc_score_done && kv->N_max > 0) {
-        dim3 sgrid((kv->N_max + kKeys - 1) / kKeys, 1, kv->P * kv->H_kv);
-        simt::score_kernel<<<sgrid, kThreads, kSmemBytes, st>>>(view, plan, q, scale_log2, ws, scores, dev_status);
-        if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
     }
     if (ev) cudaEventRecord(ev[3], st);
     return MAGE_OK;
 }
 
-static mage_status sparse_simt(const mage_kv_t *kv, const KvView &view, const Plan &plan, const __nv_bfloat16 *q,
-                               const __nv_bfloat16 *k_blk, const __nv_bfloat16 *v_blk, const int *indices,
-                               const int *k_eff, int k, float sm_scale, __nv_bfloat16 *out, float *ws, bool ws_ok,
-                               unsigned *dev_status, cudaStream_t st) {
-    using namespace simt;
-    if (!(kv->flags & MAGE_FLAG_SIMT_KERNELS) && tc::encode_fn() != nullptr) {
-        tc::AttnMaps maps;
-        auto kern_tc = tc::attn_kernel<true>;
-        if (tc::make_group_rows_map(&maps.q, q, (long long)kv->P * kv->H_kv, kv->H_q / kv->H_kv * kv->B) && opt_in_smem(kern_tc, tc::kAttnSmemBytesSparse) == MAGE_OK) {
-            maps.k = maps.v = maps.kb = maps.vb = maps.q;     // placeholders unless the TMA row gather below applies
-            long long c_rows = 0, c_pitch = 0;
-            const long long b_rows = (long long)kv->P * kv->H_kv * kv->B;
-            if (tc::eligible(kv) && tc::cache_as_rows(kv, &c_rows, &c_pitch) && tc::make_row_gather_map(&maps.k, kv->k_cache, c_rows, c_pitch) &&
-                tc::make_row_gather_map(&maps.v, kv->v_cache, c_rows, c_pitch) && tc::make_row_gather_map(&maps.kb, k_blk, b_rows, kD) &&
-                tc::make_row_gather_map(&maps.vb, v_blk, b_rows, kD) && !((reinterpret_cast<uintptr_t>(k_blk) | reinterpret_cast<uintptr_t>(v_blk)) & 15)) {
-                maps.gather_rows = (int)c_rows;
-                maps.gather_blk_rows = (int)b_rows;
-                maps.gather_pitch = (int)c_pitch;
-            }
-            const int n_rg = (view.M + 255) / 256, heads = kv->P * kv->H_kv;
-            // few (head, row-group) pairs in the launch: split each head's keys over several CTAs and merge
-            int n_split = 1;
-            if (ws_ok && plan.sparse_split_max > 1) {
-                n_split = 148 / (heads * n_rg);
-                const int tiles = (k + kv->B + 127) / 128;
-                if (n_split > tiles) n_split = tiles;
-                if (n_split > plan.sparse_split_max) n_split = plan.sparse_split_max;
-                if (n_split < 1) n_split = 1;
-            }
-            dim3 tgrid(n_split, n_rg, heads);
-            launch_pdl(kern_tc, tgrid, dim3(416), tc::kAttnSmemBytesSparse, st, maps, view, plan, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, ws, out, dev_status);
-            if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
-            if (n_split > 1) {
-                const int rows_total = heads * view.M;
-                launch_pdl(tc::sparse_combine_kernel, dim3((rows_total + 3) / 4), dim3(128), 0, st, view, plan, n_split, k, k_eff, (const float *)ws, out);
-                return launch_check();
-            }
-            return MAGE_OK;
-        }
+// Reuse step (Algorithm 1, Phase 2).
+static mage_status launch_sparse_step(const mage_kv_t *kv, const KvView &view, const Plan &plan, const __nv_bfloat16 *q,
+                                      const __nv_bfloat16 *k_blk, const __nv_bfloat16 *v_blk, const int *indices,
+                                      const int *k_eff, int k, float sm_scale, __nv_bfloat16 *out, float *ws, bool ws_ok,
+                                      unsigned *dev_status, cudaStream_t st) {
+    const int heads = kv->P * kv->H_kv;
+    if (kv->flags & MAGE_FLAG_SIMT_KERNELS) {
+        using namespace simt;
+        auto kern = attn_kernel<Mode::kSparseFinal>;
+        if (opt_in_smem(kern, kSmemBytes) != MAGE_OK) return MAGE_ERR_CUDA;
+        kern<<<dim3((view.M + kRows - 1) / kRows, 1, heads), kThreads, kSmemBytes, st>>>(view, plan, q, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, nullptr, out, dev_status);
+        return launch_check();
     }
-    auto kern = attn_kernel<Mode::kSparseFinal>;
-    if (opt_in_smem(kern, kSmemBytes) != MAGE_OK) return MAGE_ERR_CUDA;
-    dim3 grid((view.M + kRows - 1) / kRows, 1, kv->P * kv->H_kv);
-    kern<<<grid, kThreads, kSmemBytes, st>>>(view, plan, q, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, nullptr, out, dev_status);
-    return launch_check();
+    if (tc::encode_fn() == nullptr) return MAGE_ERR_CUDA;
+    tc::AttnMaps maps;
+    auto kern_tc = tc::attn_kernel<true>;
+    if (!tc::make_group_rows_map(&maps.q, q, heads, view.M)) return MAGE_ERR_UNSUPPORTED;
+    maps.k = maps.v = maps.kb = maps.vb = maps.q;         // placeholders unless the TMA row gather below applies
+    // Two gathers inside the one kernel: single 256-byte rows by TMA when the cache is one list of rows with a single pitch
+    // (every paged pool; contiguous layouts whose head and problem strides are multiples of the row stride), otherwise
+    // 16-byte cp.async, which addresses rows through 32-bit offsets in 16-byte units.
+    long long c_rows = 0, c_pitch = 0;
+    const long long b_rows = (long long)heads * kv->B;
+    const bool aligned = !((reinterpret_cast<uintptr_t>(kv->k_cache) | reinterpret_cast<uintptr_t>(kv->v_cache) | reinterpret_cast<uintptr_t>(k_blk) |
+                            reinterpret_cast<uintptr_t>(v_blk)) & 15);
+    if (kv->N_max > 0 && aligned && tc::cache_as_rows(kv, &c_rows, &c_pitch) && tc::make_row_gather_map(&maps.k, kv->k_cache, c_rows, c_pitch) &&
+        tc::make_row_gather_map(&maps.v, kv->v_cache, c_rows, c_pitch) && tc::make_row_gather_map(&maps.kb, k_blk, b_rows, kD) &&
+        tc::make_row_gather_map(&maps.vb, v_blk, b_rows, kD)) {
+        maps.gather_rows = (int)c_rows;
+        maps.gather_blk_rows = (int)b_rows;
+        maps.gather_pitch = (int)c_pitch;
+    } else {
+        if (!aligned) return MAGE_ERR_UNSUPPORTED;        // cp.async moves 16-byte pieces
+        const long long last = kv->page_size ? (long long)kv->num_pages * kv->H_kv * kv->page_size * kD
+                                             : (long long)(kv->P - 1) * kv->stride_p + (long long)(kv->H_kv - 1) * kv->stride_h + (long long)kv->N_max * kv->stride_n;
+        if ((last >> 3) > 0x7fffffffLL) return MAGE_ERR_UNSUPPORTED;
+    }
+    if (opt_in_smem(kern_tc, tc::kAttnSmemBytesSparse) != MAGE_OK) return MAGE_ERR_CUDA;
+    const int n_rg = (view.M + 255) / 256;
+    // few (head, row-group) pairs in the launch: split each head's keys over several CTAs and merge
+    int n_split = 1;
+    if (ws_ok && plan.sparse_split_max > 1) {
+        n_split = 148 / (heads * n_rg);
+        const int tiles = (k + kv->B + 127) / 128;
+        if (n_split > tiles) n_split = tiles;
+        if (n_split > plan.sparse_split_max) n_split = plan.sparse_split_max;
+        if (n_split < 1) n_split = 1;
+    }
+    launch_pdl(kern_tc, dim3(n_split, n_rg, heads), dim3(416), tc::kAttnSmemBytesSparse, st, maps, view, plan, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, ws, out, dev_status);
+    if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    if (n_split > 1) {
+        launch_pdl(tc::sparse_combine_kernel, dim3((heads * view.M + 3) / 4), dim3(128), 0, st, view, plan, n_split, k, k_eff, (const float *)ws, out);
+        return launch_check();
+    }
+    return MAGE_OK;
 }
 
 }  // namespace mage
@@ -284,7 +310,7 @@ mage_status mage_exact_select_events(const mage_kv_t *kv, const void *q, const v
     const Plan plan = make_plan(kv);
     if (workspace_bytes < plan.exact_bytes) return MAGE_ERR_WORKSPACE;
     const KvView view = make_view(kv);
-    return exact_select_simt(kv, view, plan, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_blk),
+    return launch_exact_select(kv, view, plan, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_blk),
                              static_cast<const __nv_bfloat16 *>(v_blk), sm_scale, static_cast<__nv_bfloat16 *>(out), scores,
                              static_cast<float *>(workspace), dev_status, static_cast<cudaStream_t>(stream),
                              reinterpret_cast<cudaEvent_t *>(events));
@@ -306,7 +332,7 @@ mage_status mage_exact_attn(const mage_kv_t *kv, const void *q, const void *k_bl
     const Plan plan = make_plan(kv);
     if (workspace_bytes < plan.exact_bytes) return MAGE_ERR_WORKSPACE;
     const KvView view = make_view(kv);
-    return exact_select_simt(kv, view, plan, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_blk),
+    return launch_exact_select(kv, view, plan, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_blk),
                              static_cast<const __nv_bfloat16 *>(v_blk), sm_scale, static_cast<__nv_bfloat16 *>(out), nullptr,
                              static_cast<float *>(workspace), dev_status, static_cast<cudaStream_t>(stream), nullptr);
 }
@@ -321,7 +347,7 @@ mage_status mage_select_scores(const mage_kv_t *kv, const void *q, float sm_scal
     if (workspace_bytes < plan.exact_bytes) return MAGE_ERR_WORKSPACE;
     if (kv->N_max == 0) return MAGE_OK;                   // no prefix: no score to write
     const KvView view = make_view(kv);
-    return exact_select_simt(kv, view, plan, static_cast<const __nv_bfloat16 *>(q), nullptr, nullptr, sm_scale, nullptr, scores,
+    return launch_exact_select(kv, view, plan, static_cast<const __nv_bfloat16 *>(q), nullptr, nullptr, sm_scale, nullptr, scores,
                              static_cast<float *>(workspace), dev_status, static_cast<cudaStream_t>(stream), nullptr, true);
 }
 
@@ -343,7 +369,7 @@ mage_status mage_sparse_block_attn(const mage_kv_t *kv, const void *q, const voi
     const Plan plan = make_plan(kv, k);
     const KvView view = make_view(kv);
     const bool ws_ok = workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255) && workspace_bytes >= plan.total_bytes;
-    return sparse_simt(kv, view, plan, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_blk),
+    return launch_sparse_step(kv, view, plan, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_blk),
                        static_cast<const __nv_bfloat16 *>(v_blk), indices, k_eff, k, sm_scale, static_cast<__nv_bfloat16 *>(out),
                        static_cast<float *>(workspace), ws_ok, dev_status, static_cast<cudaStream_t>(stream));
 }
@@ -366,7 +392,8 @@ mage_status mage_append_block(const mage_kv_t *kv, const void *k_blk, const void
 // Scratch for mage_exact_select_static.  In host code this name is only a handle for the runtime, not a device
 // address: the address is looked up once per device below and that pointer is what the kernels receive.
 static __device__ __align__(256) unsigned char g_static_scratch[MAGE_STATIC_SCRATCH_BYTES];
-static void *g_static_scratch_addr[64] = {};
+static void *g_static_scratch_addr[64] = {};      // per device, guarded by g_static_scratch_mu
+static std::mutex g_static_scratch_mu;
 
 mage_status mage_exact_select_static(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk,
                                      float sm_scale, void *out, float *scores, uint32_t *dev_status, void *stream) {
@@ -380,17 +407,22 @@ mage_status mage_exact_select_static(const mage_kv_t *kv, const void *q, const v
     }
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MAGE_ERR_CUDA;
-    if (!g_static_scratch_addr[dev]) {      // set-up, once per device, with that device current
-        void *addr = nullptr;
-        const cudaError_t e = cudaGetSymbolAddress(&addr, g_static_scratch);
-        if (e != cudaSuccess || !addr) {
-            std::fprintf(stderr, "libmage: cudaGetSymbolAddress(static scratch) failed: %s\n", cudaGetErrorString(e));
-            return MAGE_ERR_CUDA;
+    void *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_scratch_mu);
+        if (!g_static_scratch_addr[dev]) {  // set-up, once per device, with that device current
+            void *addr = nullptr;
+            const cudaError_t e = cudaGetSymbolAddress(&addr, g_static_scratch);
+            if (e != cudaSuccess || !addr) {
+                std::fprintf(stderr, "libmage: cudaGetSymbolAddress(static scratch) failed: %s\n", cudaGetErrorString(e));
+                return MAGE_ERR_CUDA;
+            }
+            g_static_scratch_addr[dev] = addr;
         }
-        g_static_scratch_addr[dev] = addr;
+        scratch = g_static_scratch_addr[dev];
     }
-    return mage_exact_select_events(kv, q, k_blk, v_blk, sm_scale, out, scores, g_static_scratch_addr[dev],
-                                    (size_t)MAGE_STATIC_SCRATCH_BYTES, dev_status, stream, nullptr);
+    return mage_exact_select_events(kv, q, k_blk, v_blk, sm_scale, out, scores, scratch, (size_t)MAGE_STATIC_SCRATCH_BYTES,
+                                    dev_status, stream, nullptr);
 }
 
 const char *mage_status_string(mage_status s) {

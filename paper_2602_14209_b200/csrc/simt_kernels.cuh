@@ -204,6 +204,7 @@ __global__ void __launch_bounds__(kThreads) score_kernel(KvView kv, Plan plan, c
                                                          float *__restrict__ scores, unsigned *status) {
     extern __shared__ __align__(16) float smem[];
     float *Qs = smem, *Ks = Qs + kD * kRows, *red = Ks + kD * kKeys;   // red: [16][64]
+    __shared__ int key_bad[kKeys];
     const int j0 = blockIdx.x * kKeys, z = blockIdx.z, p = z / kv.H_kv, h = z % kv.H_kv;
     const int N = seq_len_of(kv, p);
     if (j0 >= N) return;
@@ -213,6 +214,7 @@ __global__ void __launch_bounds__(kThreads) score_kernel(KvView kv, Plan plan, c
         float kvals[32];
         long long off = -1;
         if (j < N) off = cache_row_offset(kv, p, h, j, status);
+        if (quarter == 0) key_bad[key] = j < N && off < 0;    // page id out of range: the key is skipped, its score is 0
         if (off >= 0) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) bf16x8_to_float(reinterpret_cast<const uint4 *>(kv.k + off + quarter * 32)[i], kvals + 8 * i);
@@ -248,7 +250,7 @@ __global__ void __launch_bounds__(kThreads) score_kernel(KvView kv, Plan plan, c
     if (t < kKeys && j0 + t < N) {
         float acc = 0.f;
         for (int y = 0; y < 16; ++y) acc += red[y * kKeys + t];
-        scores[(size_t)z * kv.N_max + j0 + t] = acc / (float)kv.M;
+        scores[(size_t)z * kv.N_max + j0 + t] = key_bad[t] ? 0.f : acc / (float)kv.M;
     }
 }
 

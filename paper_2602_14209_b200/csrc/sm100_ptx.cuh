@@ -272,51 +272,6 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
     return r;
 }
-// 2^x for NP pairs of values without the special-function unit, so that it can run beside ex2() on other elements:
-// clamp to >= -126, round to the nearest integer n by adding 1.5*2^23, evaluate a degree-5 minimax polynomial of
-// 2^f on f = x - n in [-0.5, 0.5] (relative error 2.4e-7, the same as ex2.approx), add n to the exponent field.
-// Written stage by stage so that the NP dependency chains are interleaved in program order.  On B200 this route
-// costs ~13 issue cycles per element against 8 cycles of MUFU, so it only pays for a minority of the elements.
-template <int NP>
-__device__ __forceinline__ void ex2_poly2_n(uint64_t (&x)[NP]) {
-    const float kMagic = 12582912.f;
-    const uint64_t magic = pack2(kMagic, kMagic), neg_magic = pack2(-kMagic, -kMagic), neg_one = pack2(-1.f, -1.f);
-    uint64_t t[NP], p[NP];
-#pragma unroll
-    for (int i = 0; i < NP; ++i) {
-        float a, b;
-        unpack2(x[i], a, b);
-        x[i] = pack2(fmaxf(a, -126.f), fmaxf(b, -126.f));
-    }
-#pragma unroll
-    for (int i = 0; i < NP; ++i) t[i] = add2(x[i], magic);
-#pragma unroll
-    for (int i = 0; i < NP; ++i) p[i] = add2(t[i], neg_magic);
-#pragma unroll
-    for (int i = 0; i < NP; ++i) x[i] = fma2(p[i], neg_one, x[i]);          // f = x - n
-    const uint64_t c5 = pack2(0.0013276466634124517f, 0.0013276466634124517f), c4 = pack2(0.009675540961325169f, 0.009675540961325169f),
-                   c3 = pack2(0.05550713464617729f, 0.05550713464617729f), c2 = pack2(0.24022120237350464f, 0.24022120237350464f),
-                   c1 = pack2(0.6931469440460205f, 0.6931469440460205f), c0 = pack2(1.0000001192092896f, 1.0000001192092896f);
-#pragma unroll
-    for (int i = 0; i < NP; ++i) p[i] = fma2(c5, x[i], c4);
-#pragma unroll
-    for (int i = 0; i < NP; ++i) p[i] = fma2(p[i], x[i], c3);
-#pragma unroll
-    for (int i = 0; i < NP; ++i) p[i] = fma2(p[i], x[i], c2);
-#pragma unroll
-    for (int i = 0; i < NP; ++i) p[i] = fma2(p[i], x[i], c1);
-#pragma unroll
-    for (int i = 0; i < NP; ++i) p[i] = fma2(p[i], x[i], c0);
-#pragma unroll
-    for (int i = 0; i < NP; ++i) {
-        float p0, p1, t0, t1;
-        unpack2(p[i], p0, p1);
-        unpack2(t[i], t0, t1);
-        p0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
-        p1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
-        x[i] = pack2(p0, p1);
-    }
-}
 template <int NP>
 __device__ __forceinline__ void ex2_mufu2_n(uint64_t (&x)[NP]) {
     float a[NP], b[NP];

@@ -83,15 +83,6 @@ inline bool make_cache_map(CUtensorMap *m, const mage_kv_t *kv, const void *base
     return make_map(m, base, 4, dims, str);
 }
 
-// Whether the tensor-core kernels cover this cache description.
-inline bool eligible(const mage_kv_t *kv) {
-    if (kv->flags & MAGE_FLAG_SIMT_KERNELS) return false;
-    if (kv->N_max < 1) return false;
-    if (kv->page_size != 0 && kv->page_size % 64 != 0) return false;
-    if ((reinterpret_cast<uintptr_t>(kv->k_cache) | reinterpret_cast<uintptr_t>(kv->v_cache)) & 15) return false;
-    return encode_fn() != nullptr;
-}
-
 // Key tiles per CTA of the score pass.  One CTA per SM at a time, so the pass lasts about ceil(heads * c / 148)
 // rounds of (tiles per CTA + a fixed start cost of about three tile times: the query tile, the row statistics, the
 // first key tile); take the number of pieces per head c that minimises that.  Paged pools (sequences of different

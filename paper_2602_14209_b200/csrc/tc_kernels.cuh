@@ -18,14 +18,16 @@ constexpr int kHalfBytes = kTile * 128;    // 128 rows x 128 bytes: one d-half o
 constexpr int kTileBytes = 2 * kHalfBytes; // 32 KB
 
 // Coordinates (c1, c2, c3) of the 64-row TMA box that starts at logical cache position j (a multiple of 64).
-// Positions at or beyond N map to an out-of-range box, which TMA fills with zeros.
-__device__ __forceinline__ void cache_box_coords(const KvView &kv, int p, int h, int j, int N, int &c1, int &c2, int &c3,
+// Positions at or beyond N map to an out-of-range box, which TMA fills with zeros.  Returns true when the box lies
+// inside the prefix but its page id is out of range: the box is zero-filled too, the status bit is raised, and the
+// caller has to leave its 64 keys out of the softmax (a skipped key is not a key with logit 0).
+__device__ __forceinline__ bool cache_box_coords(const KvView &kv, int p, int h, int j, int N, int &c1, int &c2, int &c3,
                                                  unsigned *status) {
     if (kv.page_size == 0) {
         c1 = j < N ? j : kv.N_max + 64;
         c2 = h;
         c3 = p;
-        return;
+        return false;
     }
     c1 = j % kv.page_size;
     c2 = h;
@@ -33,8 +35,12 @@ __device__ __forceinline__ void cache_box_coords(const KvView &kv, int p, int h,
     if (j < N) {
         const int page = kv.block_table[(long long)p * kv.max_pages + j / kv.page_size];
         if (page >= 0 && page < kv.num_pages) c3 = page;
-        else if (status) atomicOr(status, MAGE_DEV_BAD_PAGE);
+        else {
+            if (status) atomicOr(status, MAGE_DEV_BAD_PAGE);
+            return true;
+        }
     }
+    return false;
 }
 
 // ------------------------------------------------------------------------------------------------------------
@@ -56,7 +62,7 @@ constexpr int kScoreWgs = 4;
 constexpr int kScoreThreads = kScoreWgs * 128 + 64;
 constexpr int kScoreProducerWarp = kScoreWgs * 4, kScoreMmaWarp = kScoreWgs * 4 + 1;
 constexpr int kScoreQBytes = 2 * 256 * 128;           // up to 256 query rows, two d-halves
-constexpr size_t kScoreSmemBytes = 1024 + kScoreQBytes + kScoreStages * kTileBytes + (256 + 2 * 128) * sizeof(float) + 256;
+constexpr size_t kScoreSmemBytes = 1024 + kScoreQBytes + kScoreStages * kTileBytes + (256 + 2 * 128) * sizeof(float) + 320;
 
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, KvView kv, Plan plan,
@@ -82,6 +88,9 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
            P_FULL = T_EMPTY + 4, P_EMPTY = P_FULL + 2, N_BARS = P_EMPTY + 2 };
     uint32_t *tmem_ptr_s = reinterpret_cast<uint32_t *>(bars + N_BARS);
     volatile int *abort_s = reinterpret_cast<volatile int *>(tmem_ptr_s + 1);
+    // per key tile (ring of 16, far deeper than the producer can run ahead): bit kh set = the 64-key box kh of the tile
+    // came from a page id out of range; its keys get score 0
+    volatile int *tile_bad_s = reinterpret_cast<volatile int *>(tmem_ptr_s + 2);
     auto bar = [&](int i) { return smem_u32(bars + i); };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -90,6 +99,7 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
     const int rows_lo = min(rows, (((rows + 1) >> 1) + 7) & ~7), rows_hi = rows - rows_lo;
     const int n_units = rows_hi > 0 ? 2 : 1;           // units per tile
 
+    if (tid < 16) tile_bad_s[tid] = 0;
     if (tid == 0) {
         *abort_s = 0;
         mbar_init(bar(Q_FULL), 1);
@@ -118,14 +128,15 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
             for (int i = 0; i < n_my; ++i) {
                 const int slot = i % kScoreStages, u = i / kScoreStages;
                 if (!mbar_wait(bar(EMPTY + slot), (u & 1) ^ 1, abort_s, status)) break;
-                mbar_arrive_expect_tx(bar(FULL + slot), kTileBytes);
                 const int j0 = (tile0 + i) * kTile;
-                for (int kh = 0; kh < 2; ++kh) {
-                    int c1, c2, c3;
-                    cache_box_coords(kv, p, h, j0 + kh * 64, N, c1, c2, c3, status);
+                int c1[2], c2[2], c3[2], bad = 0;
+                for (int kh = 0; kh < 2; ++kh)
+                    if (cache_box_coords(kv, p, h, j0 + kh * 64, N, c1[kh], c2[kh], c3[kh], status)) bad |= 1 << kh;
+                if (kv.page_size != 0) tile_bad_s[i & 15] = bad;       // ordered before the tile's FULL phase by the arrive below
+                mbar_arrive_expect_tx(bar(FULL + slot), kTileBytes);
+                for (int kh = 0; kh < 2; ++kh)
                     for (int dh = 0; dh < 2; ++dh)
-                        tma_load_4d(smem_u32(k_s + slot * kTileBytes + dh * kHalfBytes + kh * kBoxBytes), &map_k, bar(FULL + slot), dh * 64, c1, c2, c3);
-                }
+                        tma_load_4d(smem_u32(k_s + slot * kTileBytes + dh * kHalfBytes + kh * kBoxBytes), &map_k, bar(FULL + slot), dh * 64, c1[kh], c2[kh], c3[kh]);
                 issued = i + 1;
             }
             if (*abort_s) {   // give the copies already in flight a bounded chance to land before the CTA exits
@@ -170,15 +181,17 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
         const uint32_t taddr = tmem_base + wg * 128 + ((uint32_t)(w4 * 32) << 16);
         float prev_sum = 0.f;
         int prev_tile = -1;
-        // row half 0: add the other half's partial sum of tile t to its own and store the score
-        auto finish = [&](int t, float own) -> bool {
+        bool prev_bad = false;
+        // row half 0: add the other half's partial sum of tile t to its own and store the score (0 for a key whose page
+        // id was out of range: it is skipped by the attention pass, so it carries no probability)
+        auto finish = [&](int t, float own, bool bad) -> bool {
             float v = own;
             if (n_units == 2) {
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(P_FULL + par), (t >> 1) & 1, abort_s, status))) return false;
                 v += part_s[par * 128 + key];
                 mbar_arrive_warp(bar(P_EMPTY + par));
             }
-            v *= inv_m;
+            v = bad ? 0.f : v * inv_m;
             const int j = (tile0 + t) * kTile + key;
             if (j < N) srow[j] = accumulate ? srow[j] + v : v;
             return true;
@@ -189,6 +202,7 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                 const int use = i >> 1;
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(T_FULL + wg), use & 1, abort_s, status))) { ok = false; break; }
                 tc_fence_after_sync();
+                const bool key_bad = (tile_bad_s[i & 15] >> (key >> 6)) & 1;
                 float tail = 0.f;
                 uint64_t acc_a = pack2(0.f, 0.f), acc_b = acc_a;
                 // one step = 8 columns = 4 pairs; the TMEM load of the next step is in flight while this one is processed
@@ -273,12 +287,13 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                     mbar_arrive_warp(bar(P_FULL + par));
                 } else {
                     // finish the previous tile of this parity now, one unit late, so this warpgroup never waits for its partner
-                    if (prev_tile >= 0 && !finish(prev_tile, prev_sum)) { ok = false; break; }
+                    if (prev_tile >= 0 && !finish(prev_tile, prev_sum, prev_bad)) { ok = false; break; }
                     prev_sum = sum;
                     prev_tile = i;
+                    prev_bad = key_bad;
                 }
             }
-            if (ok && rh == 0 && prev_tile >= 0) finish(prev_tile, prev_sum);
+            if (ok && rh == 0 && prev_tile >= 0) finish(prev_tile, prev_sum, prev_bad);
         }
     }
     tc_fence_before_sync();
@@ -314,6 +329,30 @@ constexpr int kAttnQBytes = 2 * kTileBytes;            // two M-tiles of 128 row
 constexpr size_t kAttnSmemBytesDense = 1024 + kAttnQBytes + kAttnSlotsDense * kTileBytes + 512;
 constexpr size_t kAttnSmemBytesSparse = 1024 + kAttnQBytes + kAttnSlotsSparse * kTileBytes + 512 + kSparseTableCap * sizeof(int);
 constexpr float kRescaleThreshold = 8.f;               // log2 units
+
+// Reuse step, error path only: bits of the 32 selected keys from list position t0 on that must be left out of the softmax
+// (index outside the prefix, or its page id out of range).  row_tab: the CTA's table of resolved rows (-1 = left out), or
+// null when the budget exceeds the table; then idx (this head's index list, already shifted to the CTA's first key) and
+// the problem's row of the page table are consulted.  Kept out of line: the hot loops must not pay registers for it.
+__device__ __noinline__ uint32_t sparse_bad_cols(const int *row_tab, const int *idx, int t0, int n_cache, int N,
+                                                 const int *table_row, int page_size, int num_pages) {
+    uint32_t badm = 0;
+    for (int e = 0; e < 32 && t0 + e < n_cache; ++e) {
+        bool b;
+        if (row_tab) {
+            b = row_tab[t0 + e] < 0;
+        } else {
+            const int j = idx[t0 + e];
+            b = j < 0 || j >= N;
+            if (!b && page_size) {
+                const int pg = table_row[j / page_size];
+                b = pg < 0 || pg >= num_pages;
+            }
+        }
+        if (b) badm |= 1u << e;
+    }
+    return badm;
+}
 
 // gather_rows > 0 (reuse step only): k, v, kb, vb are flat row lists (pitch gather_pitch elements) with 64 x 1 boxes.
 // lse_only (exact pass only): the select stream's own pass -- row maxima and sums over the prefix, no V, no P V, no O.
@@ -377,12 +416,18 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
            PVH_DONE = P_FULL + 2, O_DONE = PVH_DONE + 2, PUB = O_DONE + 1, N_BARS = PUB + 1 };
     uint32_t *tmem_ptr_s = reinterpret_cast<uint32_t *>(bars + N_BARS);
     volatile int *abort_s = reinterpret_cast<volatile int *>(tmem_ptr_s + 1);
-    int *row_tab = reinterpret_cast<int *>(tmem_ptr_s + 4);     // SPARSE: cache offset / 8 of each selected row, -1 = skip
+    // Keys that must be left out of the softmax although their rows arrive as zeros.  SPARSE: `any_bad` below, one flag for
+    // the CTA, set when any selected index or its page is out of range (every tile then takes the careful path and looks
+    // its columns up).  DENSE: per key tile (ring of 8), bit kh set = the 64-key box kh of the tile came from a page id out
+    // of range.
+    volatile int *tile_bad_s = reinterpret_cast<volatile int *>(tmem_ptr_s + 4);
+    int *row_tab = reinterpret_cast<int *>(tmem_ptr_s + 12);    // SPARSE: cache offset / 8 of each selected row, -1 = skip
     auto bar = [&](int i) { return smem_u32(bars + i); };
     auto slot_of = [](int L) { return L % kAttnSlots; };
     auto par_of = [](int L) { return (L / kAttnSlots) & 1; };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid < 8) tile_bad_s[tid] = 0;
     if (tid == 0) {
         *abort_s = 0;
         mbar_init(bar(Q_FULL), 1);
@@ -411,10 +456,16 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
         return maps.gather_rows > 0 ? (int)(off / maps.gather_pitch) : (int)(off >> 3);
     };
     const bool use_tab = SPARSE && n_cache <= kSparseTableCap;
-    if (use_tab)
-        for (int t = tid; t < n_cache; t += blockDim.x) row_tab[t] = resolve(t);
+    int my_bad = 0;
+    if (SPARSE) {
+        for (int t = tid; t < n_cache; t += blockDim.x) {
+            const int o = resolve(t);
+            if (use_tab) row_tab[t] = o;
+            if (o < 0) my_bad = 1;
+        }
+    }
     tc_fence_before_sync();
-    __syncthreads();
+    const int any_bad = __syncthreads_or(my_bad);
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_ptr_s;
 
@@ -434,14 +485,18 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                         issued = L + 1;
                         continue;
                     }
+                    int c1[2], c2[2], c3[2], bad = 0;
+                    if (!blk_chunk) {
+                        for (int kh = 0; kh < 2; ++kh)
+                            if (cache_box_coords(kv, p, h, j_begin + i * kTile + kh * 64, N, c1[kh], c2[kh], c3[kh], is_v ? nullptr : status)) bad |= 1 << kh;
+                        if (kv.page_size != 0 && !is_v) tile_bad_s[i & 7] = bad;    // ordered before K(i)'s FULL phase by the arrive below
+                    }
                     mbar_arrive_expect_tx(bar(FULL + slot), kTileBytes);
                     const uint32_t dst = smem_u32(kv_s + slot * kTileBytes);
                     for (int kh = 0; kh < 2; ++kh) {
                         if (!blk_chunk) {
-                            int c1, c2, c3;
-                            cache_box_coords(kv, p, h, j_begin + i * kTile + kh * 64, N, c1, c2, c3, is_v ? nullptr : status);
                             for (int dh = 0; dh < 2; ++dh)
-                                tma_load_4d(dst + dh * kHalfBytes + kh * kBoxBytes, is_v ? &maps.v : &maps.k, bar(FULL + slot), dh * 64, c1, c2, c3);
+                                tma_load_4d(dst + dh * kHalfBytes + kh * kBoxBytes, is_v ? &maps.v : &maps.k, bar(FULL + slot), dh * 64, c1[kh], c2[kh], c3[kh]);
                         } else {
                             const int row = (i == 0 && kh == 0) ? z * kv.B : blk_rows_total + 64;   // beyond the tensor: zero fill
                             for (int dh = 0; dh < 2; ++dh)
@@ -716,6 +771,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 // phase of the "first half of PV accumulated" barrier before this tile's P exists (see the recovery path)
                 const uint32_t pvh_cur = mbar_test_wait(bar(PVH_DONE + mt), 0) ? 1u : 0u;
                 const int valid = min(kTile, n_keys - i * kTile);
+                const int bad = SPARSE ? any_bad : tile_bad_s[i & 7];    // (rare) keys of this tile to leave out
                 // Rescale O by f (rows that do not need it pass f = 1): no MMA touches this O between "S(i) complete"
                 // (which implies PV(i-1) complete) and "P(i) ready".
                 auto rescale_o = [&](float f) {
@@ -731,7 +787,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     tmem_wait_st();
                 };
                 // a warp whose 32 rows all lie beyond M (row padding of the last M-tile) only takes part in the hand-offs
-                bool fast = i > first && valid == kTile, half_done = false;
+                bool fast = i > first && valid == kTile && bad == 0, half_done = false;
                 if (warp_has_rows && fast) {
                     // ---- common case: one sweep over S with the reference maximum carried over from earlier tiles.
                     // exp2(x - m_used) stays representable as long as x - m_used < 100, so the true maximum is only
@@ -841,22 +897,37 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 if (warp_has_rows && !fast) {
                     // ---- careful path (first tile, ragged last tile, or a jump of the maximum by more than 2^100):
                     // find the tile's maximum first, move the reference if it grew, then exponentiate.
+                    // bits of the 32 columns from c0 on that take part: inside the tile's valid keys and not left out
+                    auto cols_ok = [&](int c0) -> uint32_t {
+                        uint32_t okm = valid - c0 >= 32 ? 0xffffffffu : (valid - c0 <= 0 ? 0u : (1u << (valid - c0)) - 1u);
+                        if (bad) {
+                            if (!SPARSE) {
+                                if ((bad >> (c0 >> 6)) & 1) okm = 0u;
+                            } else {
+                                okm &= ~sparse_bad_cols(use_tab ? row_tab : nullptr, indices + (long long)z * k + key_off, i * kTile + c0, n_cache, N,
+                                                        kv.page_size ? kv.block_table + (long long)p * kv.max_pages : nullptr, kv.page_size, kv.num_pages);
+                            }
+                        }
+                        return okm;
+                    };
                     float mx = -INFINITY;
 #pragma unroll 1
                     for (int c0 = 0; c0 < kTile; c0 += 32) {
                         uint32_t r[32];
                         tmem_ld32(tS + c0, r);
                         tmem_wait_ld();
-                        if (valid == kTile) {
+                        const uint32_t okm = cols_ok(c0);
+                        if (okm == 0xffffffffu) {
 #pragma unroll
                             for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]));
                         } else {
 #pragma unroll
                             for (int e = 0; e < 32; ++e)
-                                if (c0 + e < valid) mx = fmaxf(mx, __uint_as_float(r[e]));
+                                if ((okm >> e) & 1u) mx = fmaxf(mx, __uint_as_float(r[e]));
                         }
                     }
-                    float target = mx * scale_log2;
+                    // (a tile all of whose keys are left out has no maximum: a finite stand-in far below any logit)
+                    float target = mx == -INFINITY ? -1e30f : mx * scale_log2;
                     if (pending) target = fmaxf(target, pend_m);
                     if (i == first) {
                         m_used = target;
@@ -878,13 +949,14 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                         uint32_t r[32], pk[16];
                         tmem_ld32(tS + c0, r);
                         tmem_wait_ld();
+                        const uint32_t okm = cols_ok(c0);
 #pragma unroll
                         for (int e = 0; e < 16; ++e) {
                             float p0 = ex2(fmaf(__uint_as_float(r[2 * e]), scale_log2, neg_m));
                             float p1 = ex2(fmaf(__uint_as_float(r[2 * e + 1]), scale_log2, neg_m));
-                            if (valid != kTile) {
-                                if (c0 + 2 * e >= valid) p0 = 0.f;
-                                if (c0 + 2 * e + 1 >= valid) p1 = 0.f;
+                            if (okm != 0xffffffffu) {
+                                if (!((okm >> (2 * e)) & 1u)) p0 = 0.f;
+                                if (!((okm >> (2 * e + 1)) & 1u)) p1 = 0.f;
                             }
                             l0 += p0;
                             l1 += p1;

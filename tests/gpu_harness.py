@@ -4,7 +4,9 @@ Tolerances (written here once, used by every parity test):
   attention outputs (bf16 in, fp32 accumulate, bf16 out): max-abs 1e-2, mean-abs 1e-3 against the fp64 oracle;
   top-k: the GPU set may differ from the oracle's only in positions whose oracle score lies within 1e-5
   relative of the oracle's k-th largest score; indices distinct, in range, ascending, -1 padded;
-  scores (diagnostic bound): 2e-5 relative.
+  scores: 1e-5 relative (observed: a few 1e-7; fp32 sums of ex2.approx values against the fp64 oracle).
+Adversarial logit-jump cases, where one key dominates a row while the kernel's reference maximum lags, are compared
+with the oracle rounded to bf16 under a relative bound of two bf16 ulps (see `check_problem(o_rel_bf16=...)`).
 """
 import math
 
@@ -15,7 +17,8 @@ from paper_2602_14209_b200 import binding as mb
 from paper_2602_14209_b200 import workloads as W
 from paper_2602_14209_b200.pipeline import BlockAttention
 
-O_MAX_ABS, O_MEAN_ABS, TOPK_BAND, SCORE_REL = 1e-2, 1e-3, 1e-5, 2e-5
+O_MAX_ABS, O_MEAN_ABS, TOPK_BAND, SCORE_REL = 1e-2, 1e-3, 1e-5, 1e-5
+O_REL_BF16, O_REL_FLOOR = 2.0 ** -7, 2e-3      # two bf16 ulps, plus an absolute floor for entries near zero
 
 
 def run_gpu_block(batch, w, flags=0, paged=False, k=None, steps=None):
@@ -60,9 +63,21 @@ def check_topk_band(score_ref, idx_gpu, k, N):
     return k_eff - int(chosen[ref_set].sum())                      # positions that differ (all inside the band)
 
 
+def _bf16_round(x):
+    return torch.from_numpy(np.asarray(x, dtype=np.float32)).to(torch.bfloat16).float().numpy().astype(np.float64)
+
+
 def check_problem(oracle, batch, res, w, p, heads=None, check_scores=True, sparse_steps=None, check_topk=True,
-                  o_max_abs=O_MAX_ABS):
-    """Compare problem p of a GPU run with the oracle on the listed KV heads (default: all).  Returns diagnostics."""
+                  o_rel_bf16=False):
+    """Compare problem p of a GPU run with the oracle on the listed KV heads (default: all).  Returns diagnostics.
+
+    o_rel_bf16: the max-abs bound is replaced by |gpu - bf16(oracle)| <= 2^-7 * |bf16(oracle)| + 2e-3 per element (the
+    mean-abs bound stays).  For inputs built so that outputs reach |O| ~ 4, where one bf16 ulp alone is 1.6e-2."""
+    def o_ok(err, ref):
+        if o_rel_bf16:
+            return bool((err <= O_REL_BF16 * np.abs(ref) + O_REL_FLOOR).all()) and err.mean() <= O_MEAN_ABS
+        return err.max() <= O_MAX_ABS and err.mean() <= O_MEAN_ABS
+
     G, B, k = w.G, w.B, res["k"]
     N = int(batch["seq_lens"][p])
     heads = range(w.H_kv) if heads is None else heads
@@ -74,10 +89,12 @@ def check_problem(oracle, batch, res, w, p, heads=None, check_scores=True, spars
         qs = slice(h * G, (h + 1) * G)
         Kc, Vc = f(batch["kc"][p, h:h + 1, :N]), f(batch["vc"][p, h:h + 1, :N])
         O = oracle.exact_block_attn(f(batch["q"][0, p, qs]), Kc, Vc, f(batch["kb"][0, p, h:h + 1]), f(batch["vb"][0, p, h:h + 1]))
+        if o_rel_bf16:
+            O = _bf16_round(O)
         err = np.abs(res["outs"][0][p, qs] - O)
         assert np.isfinite(res["outs"][0][p, qs]).all()
         diag["o_max"], diag["o_mean"] = max(diag["o_max"], err.max()), max(diag["o_mean"], err.mean())
-        assert err.max() <= o_max_abs and err.mean() <= O_MEAN_ABS, (p, h, err.max(), err.mean())
+        assert o_ok(err, O), (p, h, err.max(), err.mean())
         if N > 0 and check_topk:
             sc = oracle.block_score(f(batch["q"][0, p, qs]), Kc)[0]
             got = res["scores"][p, h, :N].astype(np.float64)
@@ -94,9 +111,11 @@ def check_problem(oracle, batch, res, w, p, heads=None, check_scores=True, spars
             idx = res["indices"][p, h:h + 1]
             Os = oracle.sparse_block_attn(f(batch["q"][t, p, qs]), Kc, Vc, f(batch["kb"][t, p, h:h + 1]),
                                           f(batch["vb"][t, p, h:h + 1]), idx, k_eff)
+            if o_rel_bf16:
+                Os = _bf16_round(Os)
             e = np.abs(res["outs"][t][p, qs] - Os)
             assert np.isfinite(res["outs"][t][p, qs]).all()
             diag["sp_max"], diag["sp_mean"] = max(diag["sp_max"], e.max()), max(diag["sp_mean"], e.mean())
-            assert e.max() <= o_max_abs and e.mean() <= O_MEAN_ABS, (p, h, t, e.max(), e.mean())
+            assert o_ok(e, Os), (p, h, t, e.max(), e.mean())
     assert res["status"] == 0
     return diag

@@ -194,3 +194,20 @@ def test_recall_and_planted_structure(oracle_mod):
         r = oracle_mod.recall(idx1, idx_t, k_eff)
         assert ((r > 0.3) & (r <= 1.0)).all()
     assert (oracle_mod.recall(idx1, idx1, k_eff) == 1.0).all()
+
+
+def test_recall_known_answers(oracle_mod):
+    """Eq. 3 on hand-made index sets whose overlap is known: half, none, all, and a short prefix (k_eff < k, -1 padding),
+    where the denominator is the number of entries a set actually holds."""
+    a = np.array([[0, 1, 2, 3], [0, 1, 2, 3], [5, 6, 7, 8]], dtype=np.int32)
+    b = np.array([[2, 3, 4, 5], [4, 5, 6, 7], [8, 7, 6, 5]], dtype=np.int32)
+    assert oracle_mod.recall(a, b, 4).tolist() == [0.5, 0.0, 1.0]
+    # N = 3 < k = 5: three entries per set, the rest is padding that must not count as a match
+    a = np.array([[0, 1, 2, -1, -1]], dtype=np.int32)
+    b = np.array([[1, 2, 9, -1, -1]], dtype=np.int32)
+    np.testing.assert_allclose(oracle_mod.recall(a, b, 3), [2.0 / 3.0])
+    # one shared entry of four, two KV heads with different answers
+    a = np.array([[10, 20, 30, 40], [1, 2, 3, 4]], dtype=np.int32)
+    b = np.array([[40, 50, 60, 70], [1, 2, 3, 9]], dtype=np.int32)
+    assert oracle_mod.recall(a, b, 4).tolist() == [0.25, 0.75]
+
