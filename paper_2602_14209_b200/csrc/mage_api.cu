@@ -280,7 +280,7 @@ static mage_status launch_sparse_step(const mage_kv_t *kv, const KvView &view, c
         if (n_split > plan.sparse_split_max) n_split = plan.sparse_split_max;
         if (n_split < 1) n_split = 1;
     }
-    launch_pdl(kern_tc, dim3(n_split, n_rg, heads), dim3(416), tc::kAttnSmemBytesSparse, st, maps, view, plan, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, ws, out, dev_status);
+    launch_pdl(kern_tc, dim3(n_split, n_rg, heads), dim3(tc::kSparseThreads), tc::kAttnSmemBytesSparse, st, maps, view, plan, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, ws, out, dev_status);
     if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
     if (n_split > 1) {
         launch_pdl(tc::sparse_combine_kernel, dim3((heads * view.M + 3) / 4), dim3(128), 0, st, view, plan, n_split, k, k_eff, (const float *)ws, out);
@@ -437,5 +437,9 @@ const char *mage_status_string(mage_status s) {
 }
 
 uint64_t mage_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+#ifdef MAGE_TIMING
+int mage_debug_stamps(unsigned long long *host_out) { return (int)cudaMemcpyFromSymbol(host_out, tc::g_stamps, sizeof(unsigned long long) * 128); }
+#endif
 
 }  // extern "C"

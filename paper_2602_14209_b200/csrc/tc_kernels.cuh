@@ -12,6 +12,22 @@
 namespace mage {
 namespace tc {
 
+// Development aid, compiled out of the library: with -DMAGE_TIMING, CTA (0,0,0) of the attention kernel writes
+// %globaltimer stamps at its hand-off points into a device array that mage_debug_stamps() copies out.
+#ifdef MAGE_TIMING
+__device__ unsigned long long g_stamps[128];
+__device__ __forceinline__ void stamp_at(int i) {
+    if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && i < 128) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        g_stamps[i] = t;
+    }
+}
+#define MAGE_STAMP(i) stamp_at(i)
+#else
+#define MAGE_STAMP(i) ((void)0)
+#endif
+
 constexpr int kTile = 128;                 // keys per tile
 constexpr int kBoxBytes = 64 * 128;        // one TMA box: 64 rows x 64 bf16 (128 bytes), 128-byte swizzled
 constexpr int kHalfBytes = kTile * 128;    // 128 rows x 128 bytes: one d-half of a K or V tile
@@ -329,6 +345,11 @@ constexpr int kAttnQBytes = 2 * kTileBytes;            // two M-tiles of 128 row
 constexpr size_t kAttnSmemBytesDense = 1024 + kAttnQBytes + kAttnSlotsDense * kTileBytes + 512;
 constexpr size_t kAttnSmemBytesSparse = 1024 + kAttnQBytes + kAttnSlotsSparse * kTileBytes + 512 + kSparseTableCap * sizeof(int);
 constexpr float kRescaleThreshold = 8.f;               // log2 units
+// Reuse step: warps that issue the row gathers.  A TMA request keeps the issuing warp for about 115 cycles whatever it
+// fetches, and the lanes of a warp issue one after the other, so the gather rate of a CTA is set by the number of warps
+// that issue: seven fill a 512-thread CTA beside the eight softmax warps and the MMA warp.
+constexpr int kSparseProducerWarps = 7;
+constexpr int kSparseThreads = 256 + kSparseProducerWarps * 32 + 32;
 
 // Reuse step, error path only: bits of the 32 selected keys from list position t0 on that must be left out of the softmax
 // (index outside the prefix, or its page id out of range).  row_tab: the CTA's table of resolved rows (-1 = left out), or
@@ -362,18 +383,21 @@ struct AttnMaps {
 };
 
 template <bool SPARSE>
-__global__ void __launch_bounds__(SPARSE ? 416 : 320, 1)
+__global__ void __launch_bounds__(SPARSE ? kSparseThreads : 320, 1)
 attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const __nv_bfloat16 *__restrict__ k_blk,
             const __nv_bfloat16 *__restrict__ v_blk, const int *__restrict__ indices, const int *__restrict__ k_eff_arr, int k,
             float scale_log2, float *__restrict__ ws, __nv_bfloat16 *__restrict__ out, unsigned *status) {
     using namespace ptx;
+    if (threadIdx.x == 0) MAGE_STAMP(0);
+    if (threadIdx.x < 5) prefetch_tensormap(&maps.q + threadIdx.x);    // (kernel parameters: no need to wait for the predecessor)
     pdl_wait();                      // everything below may read what the previous kernel in the stream wrote
     pdl_launch_dependents();
-    constexpr int kMmaWarp = SPARSE ? 12 : 9;
+    if (threadIdx.x == 0) MAGE_STAMP(1);
+    constexpr int kMmaWarp = SPARSE ? 8 + kSparseProducerWarps : 9;
     constexpr int kAttnSlots = SPARSE ? kAttnSlotsSparse : kAttnSlotsDense;
     const int chunk = blockIdx.x, rg = blockIdx.y, z = blockIdx.z, p = z / kv.H_kv, h = z % kv.H_kv;
     const int N = seq_len_of(kv, p);
-    int n_keys, n_cache, j_begin = 0;
+    int n_keys, n_cache, j_begin = 0, first_idx = 0;
     bool blk_chunk = false;
     if (!SPARSE) {
         if (chunk < plan.n_chunks) {
@@ -386,6 +410,9 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             n_cache = 0;
         }
     } else {
+        // (the thread's first selected index starts its way in before the problem's k_eff is read, so that the two cold
+        // loads overlap; the unsplit launch only, where the CTA's list starts at the head's first index)
+        if (gridDim.x == 1 && (int)threadIdx.x < k) first_idx = indices[(long long)z * k + threadIdx.x];
         n_cache = min(max(k_eff_arr[p], 0), k);
         n_keys = n_cache + kv.B;
     }
@@ -402,6 +429,9 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
         n_cache = max(0, blk_shift);
     }
     const int n_tiles = (n_keys + kTile - 1) / kTile;
+    // Reuse step: the last tile of the list usually holds little more than the block's own keys; it is gathered, multiplied
+    // and exponentiated at its own width (a multiple of 16 keys) instead of a full 128.
+    const int last_cols = SPARSE ? ((n_keys - (n_tiles - 1) * kTile + 15) & ~15) : kTile;
     const int rows_here = min(256, kv.M - rg * 256), n_mt = rows_here > 128 ? 2 : 1;
     // With a single M-tile the second softmax warpgroup and the second S/O regions would idle.  They take the
     // odd key tiles instead ("tile-parity mode"): two independent online-softmax pipelines over the same 128 rows,
@@ -431,7 +461,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
     if (tid == 0) {
         *abort_s = 0;
         mbar_init(bar(Q_FULL), 1);
-        for (int s = 0; s < kAttnSlots; ++s) { mbar_init(bar(FULL + s), SPARSE ? 4 : 1); mbar_init(bar(EMPTY + s), 1); }
+        for (int s = 0; s < kAttnSlots; ++s) { mbar_init(bar(FULL + s), SPARSE ? (maps.gather_rows > 0 ? kSparseProducerWarps : 4) : 1); mbar_init(bar(EMPTY + s), 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(S_FULL + b), 1);
             mbar_init(bar(P_HALF + b), 4);                  // one arrival per warp
@@ -441,12 +471,19 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
         mbar_init(bar(O_DONE), 1);
         mbar_init(bar(PUB), 4);
         fence_mbar_init();
+        fence_proxy_async();
+        // the queries start their way in at once: (d, row within the KV head's G*B rows, head); rows past the head read as zeros
+        mbar_arrive_expect_tx(bar(Q_FULL), n_mt * kTileBytes);
+        for (int mt = 0; mt < n_mt; ++mt)
+            for (int dh = 0; dh < 2; ++dh)
+                for (int rb = 0; rb < 2; ++rb)
+                    tma_load_3d(smem_u32(q_s + mt * kTileBytes + dh * kHalfBytes + rb * kBoxBytes), &maps.q, bar(Q_FULL), dh * 64,
+                                rg * 256 + mt * kTile + rb * 64, z);
     }
     if (warp == kMmaWarp) { tmem_alloc(smem_u32(tmem_ptr_s), 512); tmem_relinquish(); }
     // SPARSE: resolve every selected index to a cache row once (shared by the K and V gathers): bounds check,
     // page-table lookup, offset in 16-byte units.  Budgets beyond the table are resolved on the fly.
-    auto resolve = [&](int t) -> int {
-        const int j = indices[(long long)z * k + key_off + t];
+    auto resolve_idx = [&](int j) -> int {
         if (j < 0 || j >= N) {
             if (status) atomicOr(status, MAGE_DEV_BAD_INDEX);
             return -1;
@@ -455,11 +492,12 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
         if (off < 0) return -1;
         return maps.gather_rows > 0 ? (int)(off / maps.gather_pitch) : (int)(off >> 3);
     };
+    auto resolve = [&](int t) -> int { return resolve_idx(indices[(long long)z * k + key_off + t]); };
     const bool use_tab = SPARSE && n_cache <= kSparseTableCap;
     int my_bad = 0;
     if (SPARSE) {
         for (int t = tid; t < n_cache; t += blockDim.x) {
-            const int o = resolve(t);
+            const int o = gridDim.x == 1 && t == tid ? resolve_idx(first_idx) : resolve(t);
             if (use_tab) row_tab[t] = o;
             if (o < 0) my_bad = 1;
         }
@@ -467,14 +505,13 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
     tc_fence_before_sync();
     const int any_bad = __syncthreads_or(my_bad);
     tc_fence_after_sync();
+    if (threadIdx.x == 0) MAGE_STAMP(2);
     const uint32_t tmem_base = *tmem_ptr_s;
 
     if (warp >= 8 && warp != kMmaWarp) {
         // ------------------------------------------------------------------ producers
         if (!SPARSE) {
             if (lane == 0) {
-                prefetch_tensormap(blk_chunk ? &maps.kb : &maps.k);
-                prefetch_tensormap(blk_chunk ? &maps.vb : &maps.v);
                 const int blk_rows_total = kv.P * kv.H_kv * kv.B;
                 int issued = 0;
                 for (int L = 0; L < 2 * n_tiles; ++L) {
@@ -515,33 +552,51 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
         } else {
             const int pt = tid - 256, cchunk = pt & 15, r0 = pt >> 4;
             if (maps.gather_rows > 0) {
-                // TMA row gather: thread r of the 128 producers fetches row r of every tile as two 64 x 1 boxes (the two
-                // d-halves).  Unlike 16-byte cp.async, these requests do not pass through the L1 miss queue, which
-                // limits a CTA to about 17 GB/s of scattered rows.  Rows that do not exist (a bad index, the tail of
-                // the last tile) are fetched from beyond the tensor and arrive as zeros.  Each warp announces its 32 rows
-                // (8 KB) on the slot's barrier before its lanes issue.
-                if (lane == 0) {
-                    prefetch_tensormap(&maps.k); prefetch_tensormap(&maps.v); prefetch_tensormap(&maps.kb); prefetch_tensormap(&maps.vb);
-                }
+                // TMA row gather, four rows per request: the cache is one 2-D tensor of 256-byte rows with a 64 x 1 box, and a
+                // request names a column (d-half) and four row numbers, whose 128-byte halves land in four consecutive
+                // rows of the swizzled tile.  Rows that do not exist (a bad index, the tail of the last tile) are named
+                // beyond the tensor and arrive as zeros.
                 int issued = 0;
                 for (int L = 0; L < 2 * n_tiles; ++L) {
                     const int i = L >> 1, is_v = L & 1, slot = slot_of(L);
                     if (!__all_sync(0xffffffffu, mbar_wait(bar(EMPTY + slot), par_of(L) ^ 1, abort_s, status))) break;
-                    if (lane == 0) mbar_arrive_expect_tx(bar(FULL + slot), 32 * 256);
-                    __syncwarp();
-                    const int t = i * kTile + pt;
-                    const CUtensorMap *map = is_v ? &maps.v : &maps.k;
-                    int row = maps.gather_rows;                       // beyond the tensor: zero fill
-                    if (t < n_cache) {
-                        const int o = use_tab ? row_tab[t] : resolve(t);
-                        if (o >= 0) row = o;
-                    } else {
-                        map = is_v ? &maps.vb : &maps.kb;
-                        row = t < n_keys ? z * kv.B + (t - blk_shift) : maps.gather_blk_rows;
+                    // rows of this tile that are used at all (a multiple of 16), and this warp's share of them
+                    // Requests of a tile: (group of four consecutive list positions, d-half), 64 for a full tile, fewer for
+                    // the last one; request o goes to warp o % 7, lane o / 7.  Each warp announces its share of the bytes.
+                    const int pw = pt >> 5;
+                    const int n_req = ((i == n_tiles - 1 ? last_cols : kTile) >> 2) * 2;
+                    const int mine = n_req > pw ? (n_req - pw + kSparseProducerWarps - 1) / kSparseProducerWarps : 0;
+                    if (lane == 0) {
+                        if (mine > 0) mbar_arrive_expect_tx(bar(FULL + slot), mine * 512);
+                        else mbar_arrive(bar(FULL + slot));
                     }
-                    const uint32_t dst = smem_u32(kv_s + slot * kTileBytes + pt * 128);
-                    tma_load_2d(dst, map, bar(FULL + slot), 0, row);
-                    tma_load_2d(dst + kHalfBytes, map, bar(FULL + slot), 64, row);
+                    __syncwarp();
+                    if (lane < mine) {
+                        const int o = lane * kSparseProducerWarps + pw;
+                        const int r_in_tile = (o >> 1) * 4, dh = o & 1, t0 = i * kTile + r_in_tile;
+                        int rows[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int t = t0 + e;
+                            if (t < n_cache) {
+                                const int ro = use_tab ? row_tab[t] : resolve(t);
+                                rows[e] = ro >= 0 ? ro : maps.gather_rows;          // beyond the tensor: zero fill
+                            } else {
+                                rows[e] = t < n_keys ? z * kv.B + (t - blk_shift) : maps.gather_blk_rows;
+                            }
+                        }
+                        const uint32_t dst = smem_u32(kv_s + slot * kTileBytes + dh * kHalfBytes + r_in_tile * 128);
+                        if (t0 + 3 < n_cache) {
+                            tma_gather4_2d(dst, is_v ? &maps.v : &maps.k, bar(FULL + slot), dh * 64, rows[0], rows[1], rows[2], rows[3]);
+                        } else if (t0 >= n_cache) {
+                            tma_gather4_2d(dst, is_v ? &maps.vb : &maps.kb, bar(FULL + slot), dh * 64, rows[0], rows[1], rows[2], rows[3]);
+                        } else {                                                    // the group straddles the end of the selected rows
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                tma_load_2d(dst + e * 128, t0 + e < n_cache ? (is_v ? &maps.v : &maps.k) : (is_v ? &maps.vb : &maps.kb), bar(FULL + slot), dh * 64, rows[e]);
+                        }
+                    }
+                    if (tid == 256) MAGE_STAMP(40 + L);
                     issued = L + 1;
                 }
                 if (*abort_s) {                                        // let the copies in flight land before the CTA leaves
@@ -550,7 +605,8 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                         while (!mbar_try_wait(bar(FULL + slot_of(L)), par_of(L)) && clock64() - t0 < 2000000) {}
                     }
                 }
-            } else {
+            } else if (pt < 128) {
+            // (16-byte cp.async path: the first four producer warps gather, the others have nothing to do)
             // Up to three gathers are in flight and a load is posted (its FULL barrier signalled) once the two younger
             // ones have been issued -- unless the ring is full: then everything in flight is waited for and posted before
             // the warp blocks on the slot, so that the MMA side never waits for a load that has already landed.
@@ -597,14 +653,9 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issue (one lane)
         if (lane == 0) {
-            prefetch_tensormap(&maps.q);
-            mbar_arrive_expect_tx(bar(Q_FULL), n_mt * kTileBytes);
-            for (int mt = 0; mt < n_mt; ++mt)
-                for (int dh = 0; dh < 2; ++dh)
-                    for (int rb = 0; rb < 2; ++rb)     // (d, row within the KV head's G*B rows, head): rows past the head read as zeros
-                        tma_load_3d(smem_u32(q_s + mt * kTileBytes + dh * kHalfBytes + rb * kBoxBytes), &maps.q, bar(Q_FULL), dh * 64,
-                                    rg * 256 + mt * kTile + rb * 64, z);
             const uint32_t idesc_qk = idesc_bf16_f32(kTile, false, false);   // S[128 rows][128 keys]
+            const uint32_t idesc_qk_last = idesc_bf16_f32(last_cols, false, false);
+            const int nks_last = last_cols >> 4;                             // 16-key steps of the last tile's P V
             const uint32_t idesc_pv = idesc_bf16_f32(kD, false, true);       // O[128 rows][128 d], V is MN-major
             // The issuing thread runs in step with the tensor pipe (an MMA is accepted only as the previous one drains),
             // so whatever it executes between two MMAs is idle time of the pipe.  Hence: shared-memory descriptors are
@@ -629,47 +680,51 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             };
             auto ring_at = [](int L) { return Ring{L % kAttnSlots, (uint32_t)((L / kAttnSlots) & 1)}; };
             // reg = which S/O region (and softmax warpgroup); the Q tile is reg with two M-tiles, tile 0 in tile-parity mode
-            auto qk = [&](int slot, int reg) {
+            auto qk = [&](int slot, int reg, int tile) {
                 const uint32_t a0 = q_lo + (tp ? 0u : (uint32_t)reg * kTileU), b0 = k_lo + (uint32_t)slot * kTileU;
+                const uint32_t idesc = SPARSE && tile == n_tiles - 1 ? idesc_qk_last : idesc_qk;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint32_t off = (ks >> 2) * kHalfU + (ks & 3) * 2;
-                    umma_ss(tmem_base + reg * 128, desc(a0 + off), desc(b0 + off), idesc_qk, ks > 0);
+                    umma_ss(tmem_base + reg * 128, desc(a0 + off), desc(b0 + off), idesc, ks > 0);
                 }
             };
             // half 0: keys 0-63 of the tile, half 1: keys 64-127; 16 keys per step = 16 rows of 128 bytes in each d-half
-            auto pv = [&](int slot, int reg, int half, uint32_t acc) {
+            auto pv = [&](int slot, int reg, int half, uint32_t acc, int tile) {
                 if (maps.lse_only) return;
                 const uint32_t b0 = v_lo + (uint32_t)slot * kTileU;
+                const int nks = SPARSE && tile == n_tiles - 1 ? nks_last : 8;
 #pragma unroll
                 for (int ks = half * 4; ks < half * 4 + 4; ++ks)
-                    umma_ts(tmem_base + 256 + reg * 128, tmem_base + reg * 128 + ks * 8, desc(b0 + ks * (2048 >> 4)), idesc_pv, ks > 0 ? 1u : acc);
+                    if (!SPARSE || ks < nks)
+                        umma_ts(tmem_base + 256 + reg * 128, tmem_base + reg * 128 + ks * 8, desc(b0 + ks * (2048 >> 4)), idesc_pv, ks > 0 ? 1u : acc);
             };
             auto wait_full = [&](const Ring &r) { return mbar_wait(bar(FULL + r.slot), r.par, abort_s, status); };
             auto peek_p = [&](int reg, int ph) { return mbar_test_wait(bar(P_FULL + reg), ph); };
             // Looks at barriers ahead of time: the test is issued before a batch of MMAs and its result is used after it,
             // so its latency (about a hundred cycles even when the phase is complete) overlaps with the issue of the batch.
             auto peek_full = [&](const Ring &r) { return mbar_test_wait(bar(FULL + r.slot), r.par); };
-            auto pv_tile = [&](int slot, int reg, int ph, uint32_t acc, bool p_ready) -> bool {
+            auto pv_tile = [&](int slot, int reg, int ph, uint32_t acc, bool p_ready, int tile) -> bool {
                 if (p_ready || mbar_test_wait(bar(P_FULL + reg), ph)) {
                     tc_fence_after_sync();
-                    pv(slot, reg, 0, acc);
-                    pv(slot, reg, 1, acc);
+                    pv(slot, reg, 0, acc, tile);
+                    pv(slot, reg, 1, acc, tile);
                     return true;
                 }
                 if (!mbar_wait(bar(P_HALF + reg), ph, abort_s, status)) return false;
                 tc_fence_after_sync();
-                pv(slot, reg, 0, acc);
+                pv(slot, reg, 0, acc, tile);
                 umma_commit(bar(PVH_DONE + reg));
                 if (!mbar_wait(bar(P_FULL + reg), ph, abort_s, status)) return false;
                 tc_fence_after_sync();
-                pv(slot, reg, 1, acc);
+                pv(slot, reg, 1, acc, tile);
                 return true;
             };
             // The reuse step is a handful of tiles long and latency-bound: there the slots go back by commits right after
             // their last MMA, which is sooner than the softmax warpgroup's wake-up.
             constexpr bool kCommitFrees = SPARSE;
             bool ok = mbar_wait(bar(Q_FULL), 0, abort_s, status);
+            MAGE_STAMP(3);
             if (tp) {
                 // tile i belongs to pipeline i & 1; its QK^T is issued two tiles ahead, right after the PV of tile i-2
                 Ring rk = ring_at(0), rv = ring_at(1);
@@ -677,7 +732,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     ok = wait_full(rk);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    qk(rk.slot, i);
+                    qk(rk.slot, i, i);
                     umma_commit(bar(S_FULL + i));
                     if (kCommitFrees) umma_commit(bar(EMPTY + rk.slot));
                 }
@@ -685,14 +740,14 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 for (int i = 0; ok && i < n_tiles; ++i, rk.next(), rv.next()) {
                     const int reg = i & 1, ph = (i >> 1) & 1;
                     if (!wait_full(rv)) break;
-                    if (!pv_tile(rv.slot, reg, ph, i > 1 ? 1u : 0u, peek_p(reg, ph))) break;
+                    if (!pv_tile(rv.slot, reg, ph, i > 1 ? 1u : 0u, peek_p(reg, ph), i)) break;
                     // V(i) goes back by a commit of its own here: the next S of this pipeline needs K(i+2), and a gathering
                     // producer posts K(i+2) only after it has issued two more loads, the first of them into V(i)'s slot
                     umma_commit(bar(EMPTY + rv.slot));
                     if (i + 2 < n_tiles) {
                         if (!wait_full(rk)) break;
                         tc_fence_after_sync();
-                        qk(rk.slot, reg);
+                        qk(rk.slot, reg, i + 2);
                         umma_commit(bar(S_FULL + reg));
                         if (kCommitFrees) umma_commit(bar(EMPTY + rk.slot));
                     }
@@ -700,11 +755,12 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             } else {
                 Ring rk = ring_at(0), rv = ring_at(1);
                 if (ok) ok = wait_full(rk);
+                MAGE_STAMP(4);
                 if (ok) {
                     tc_fence_after_sync();
-                    qk(rk.slot, 0);
+                    qk(rk.slot, 0, 0);
                     umma_commit(bar(S_FULL + 0));
-                    qk(rk.slot, 1);
+                    qk(rk.slot, 1, 0);
                     umma_commit(bar(S_FULL + 1));
                     if (kCommitFrees) umma_commit(bar(EMPTY + rk.slot));
                 }
@@ -715,19 +771,21 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     const int ph = i & 1;
                     const uint32_t acc = i > 0 ? 1u : 0u;
                     if (!v_ready && !wait_full(rv)) break;
+                    MAGE_STAMP(80 + i);
                     // (a gathered K(i+1) may land after P(i) is ready: the reuse step does not hold PV(i) back for it)
                     if (!SPARSE && more && !k_ready && !wait_full(rk)) break;
-                    if (!pv_tile(rv.slot, 0, ph, acc, p0_ready)) break;
+                    if (!pv_tile(rv.slot, 0, ph, acc, p0_ready, i)) break;
                     const bool p1_ready = peek_p(1, ph);
                     if (more) {
                         if (SPARSE) {
                             if (!wait_full(rk)) break;
                             tc_fence_after_sync();
                         }
-                        qk(rk.slot, 0);
+                        qk(rk.slot, 0, i + 1);
                         umma_commit(bar(S_FULL + 0));
                     }
-                    if (!pv_tile(rv.slot, 1, ph, acc, p1_ready)) break;
+                    if (!pv_tile(rv.slot, 1, ph, acc, p1_ready, i)) break;
+                    MAGE_STAMP(60 + i);
                     if (kCommitFrees) umma_commit(bar(EMPTY + rv.slot));
                     if (more) {
                         Ring rv1 = rv, rk1 = rk;
@@ -736,7 +794,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                         v_ready = peek_full(rv1);
                         k_ready = i + 2 < n_tiles && peek_full(rk1);
                         p0_ready = peek_p(0, ph ^ 1);
-                        qk(rk.slot, 1);
+                        qk(rk.slot, 1, i + 1);
                         umma_commit(bar(S_FULL + 1));
                         if (kCommitFrees) umma_commit(bar(EMPTY + rk.slot));
                     }
@@ -762,6 +820,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 const int ph = (tp ? i >> 1 : i) & 1;
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(S_FULL + mt), ph, abort_s, status))) { ok = false; break; }
                 tc_fence_after_sync();
+                if (tid == 0) MAGE_STAMP(10 + 2 * i);
                 // S(i) complete means every MMA issued before it is complete too: K(i) and (two M-tiles) V(i-1), whose PV
                 // was issued just before this QK^T, have been read for the last time; their slots go back to the producer.
                 if (!SPARSE && w4 == 0 && lane == 0 && (tp || mt == 1)) {
@@ -771,6 +830,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 // phase of the "first half of PV accumulated" barrier before this tile's P exists (see the recovery path)
                 const uint32_t pvh_cur = mbar_test_wait(bar(PVH_DONE + mt), 0) ? 1u : 0u;
                 const int valid = min(kTile, n_keys - i * kTile);
+                const int cols_here = SPARSE && i == n_tiles - 1 ? ((valid + 31) & ~31) : kTile;    // columns of S in use, by 32
                 const int bad = SPARSE ? any_bad : tile_bad_s[i & 7];    // (rare) keys of this tile to leave out
                 // Rescale O by f (rows that do not need it pass f = 1): no MMA touches this O between "S(i) complete"
                 // (which implies PV(i-1) complete) and "P(i) ready".
@@ -787,7 +847,19 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     tmem_wait_st();
                 };
                 // a warp whose 32 rows all lie beyond M (row padding of the last M-tile) only takes part in the hand-offs
-                bool fast = i > first && valid == kTile && bad == 0, half_done = false;
+                bool fast = valid == kTile && bad == 0, half_done = false;
+                if (warp_has_rows && fast && i == first) {
+                    // first tile: the reference starts at the maximum of the row's first 32 logits; the sweep below moves it
+                    // on lazily like any later rise (and redoes the tile on the careful path if the rest of the row lies
+                    // more than 2^100 above it)
+                    uint32_t r0[32];
+                    tmem_ld32(tS, r0);
+                    tmem_wait_ld(r0);
+                    float m0 = __uint_as_float(r0[0]);
+#pragma unroll
+                    for (int e = 1; e < 32; ++e) m0 = fmaxf(m0, __uint_as_float(r0[e]));
+                    m_used = m0 * scale_log2;
+                }
                 if (warp_has_rows && fast) {
                     // ---- common case: one sweep over S with the reference maximum carried over from earlier tiles.
                     // exp2(x - m_used) stays representable as long as x - m_used < 100, so the true maximum is only
@@ -912,7 +984,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     };
                     float mx = -INFINITY;
 #pragma unroll 1
-                    for (int c0 = 0; c0 < kTile; c0 += 32) {
+                    for (int c0 = 0; c0 < cols_here; c0 += 32) {
                         uint32_t r[32];
                         tmem_ld32(tS + c0, r);
                         tmem_wait_ld();
@@ -945,7 +1017,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     const float neg_m = -m_used;
                     float l0 = 0.f, l1 = 0.f;
 #pragma unroll 1
-                    for (int c0 = 0; c0 < kTile; c0 += 32) {
+                    for (int c0 = 0; c0 < cols_here; c0 += 32) {
                         uint32_t r[32], pk[16];
                         tmem_ld32(tS + c0, r);
                         tmem_wait_ld();
@@ -985,6 +1057,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 tc_fence_before_sync();
                 if (!half_done) mbar_arrive_warp(bar(P_HALF + mt));
                 mbar_arrive_warp(bar(P_FULL + mt));
+                if (tid == 0) MAGE_STAMP(11 + 2 * i);
             }
             // Tile-parity mode: warpgroup 1 publishes its (reference, sum) and is done; warpgroup 0 folds the second
             // accumulator (same TMEM lanes, columns + 128) into its own while it writes the result.  The spare Q tile
@@ -1002,6 +1075,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             }
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(O_DONE), 0, abort_s, status));
             if (ok && merge) ok = __all_sync(0xffffffffu, mbar_wait(bar(PUB), 0, abort_s, status));
+            if (tid == 0) MAGE_STAMP(30);
             if (ok) {
                 tc_fence_after_sync();
                 const bool row_ok = grow < kv.M;
@@ -1090,9 +1164,11 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             }
         }
     }
+    if (tid == 0) MAGE_STAMP(31);
     tc_fence_before_sync();
     __syncthreads();
     if (warp == kMmaWarp) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
+    if (tid == 0) MAGE_STAMP(32);
 }
 
 // Merge of a reuse step that was split over n_split CTAs per KV head: one warp per query row, fixed order.
