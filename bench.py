@@ -116,6 +116,52 @@ def stage_bytes_flops(w, lens):
             "s1_flops_score": s1_flops_score, "s3_bytes": s3_bytes, "s3_flops": s3_flops}
 
 
+def config_of(w, lens, world, kernels):
+    """The `config` object of the JSON line; both arms print the same keys."""
+    return {"workload": w.name, "H_q": w.H_q, "H_kv": w.H_kv, "d": w.d, "N": w.N, "B": w.B, "k": w.k, "T": w.T,
+            "problems": w.P, "cached_tokens": sum(lens), "kv_bytes": sum(lens) * w.H_kv * 512,
+            "l2_policy": "inputs_larger_than_l2 (KV cache streamed every step evicts L2)",
+            "parallelism": f"replicas x{world} (independent blocks, no collective)", "kernels": kernels}
+
+
+def spawn_ranks_if_needed(args):
+    """`python bench.py --gpus N` (N > 1) outside torchrun: start the N ranks here, one per GPU, over 127.0.0.1."""
+    if args.gpus <= 1 or "WORLD_SIZE" in os.environ or args.impl == "reference":
+        return
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    os.execv(sys.executable, cmd)
+
+
+def bootstrap_only(args):
+    """Rank bootstrap and the max-over-ranks reduction alone (no kernels): what the N-rank launch path does around the
+    timed region.  Uses NCCL when every rank has a GPU, gloo otherwise, so it also runs on a CPU-only box."""
+    import torch
+    import torch.distributed as dist
+    rank, world, local_rank = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("LOCAL_RANK", "0"))
+    use_cuda = torch.cuda.is_available() and torch.cuda.device_count() >= world
+    if world > 1:
+        if use_cuda:
+            torch.cuda.set_device(local_rank)
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        else:
+            dist.init_process_group("gloo")
+    dev = torch.device("cuda", local_rank) if use_cuda else torch.device("cpu")
+    t = torch.tensor([float(rank + 1)], dtype=torch.float64, device=dev)      # stands in for this rank's elapsed time
+    if world > 1:
+        dist.barrier()
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    if rank == 0:
+        print(json.dumps({"bootstrap_only": True, "n_gpus": world, "max_over_ranks": float(t[0]),
+                          "backend": ("nccl" if use_cuda else "gloo") if world > 1 else None}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def run_reference(args, w):
     """The CPU oracle, as it stands, on a bounded sample: one KV head of one layer per step, scaled to the whole block."""
     import numpy as np
@@ -145,12 +191,13 @@ def run_reference(args, w):
     cores = oracle.num_threads()
     sample = (f"problem {p} (one layer/sequence, all {w.H_kv} KV heads, N={head_tokens}) of {w.name}: exact + score + top-k + "
               f"{w.T - 1} sparse steps; scaled to the whole block by cached tokens ({all_head_tokens / head_tokens:.1f}x)")
+    scale = all_head_tokens / head_tokens
     line = {"impl": "reference", "metric": METRIC, "value": ms_block, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_block, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "H_q": w.H_q, "H_kv": w.H_kv, "d": w.d, "N": w.N, "B": w.B, "k": w.k, "T": w.T, "problems": w.P},
+            "dtype": "f64", "data": "synthetic", "extrapolated": scale != 1.0, "scale": scale,
+            "config": config_of(w, lens, 1, "cpu oracle"),
             "cpu_baseline": {"value": ms_block, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
-                             "sample_seconds": per_sample},
+                             "sample_seconds": per_sample, "extrapolated": scale != 1.0, "scale": scale},
             "e2e": {"value": ms_block, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -170,8 +217,13 @@ def main():
                     help="override the lower bound of the per-sequence prefix lengths (0 = every sequence has N tokens)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-stage-breakdown", action="store_true")
+    ap.add_argument("--bootstrap-only", action="store_true", help="start the ranks, reduce a stand-in time over them and exit (no kernels)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
+    spawn_ranks_if_needed(args)
+    if args.bootstrap_only:
+        bootstrap_only(args)
+        return
 
     from paper_2602_14209_b200 import workloads as W
     w = W.CONFIGS[args.workload]
@@ -327,7 +379,7 @@ def main():
         def two_stream_phase1():
             ba.select_scores_async(q_d[0]); ba.exact_attn(q_d[0], kb_d[0], vb_d[0], outs[0]); ba.join()
 
-        sel_alone = lambda: mb.mage_select_scores(kv, q_d[0], ba.sm_scale, ba.scores, ba._select_workspace, ba.status)
+        sel_alone = lambda: mb.mage_select_scores(kv, q_d[0], ba.sm_scale, ba.scores, ba.select_workspace(), ba.status)
         two_stream_phase1(); torch.cuda.synchronize()
         p1_fused, p1_two, sel_ms = timed(fused_phase1, False, 5), timed(two_stream_phase1, False, 5), timed(sel_alone, False, 5)
         stages = {
@@ -420,26 +472,50 @@ def main():
         return
 
     # ---- roofline of the dominant kernel (the Step-1 attention kernel) -------------------------------------------
+    # Which measured bf16 peak applies depends on the regime the run was in: a short run at full clock with no power
+    # cap sampled is the burst regime; under sw_power_cap (or with the SM clock well below its maximum) the sustained one.
     attn_avg_ms = sum(attn_ms) / len(attn_ms)
+    burst_regime = (clocks.get("sm_mhz") or 0) >= 0.95 * (clocks.get("sm_max_mhz") or 1e9) and "sw_power_cap" not in clocks.get("reasons", [])
     if args.simt:
         peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
         roofline = {"bound": "alu", "kernel": "simt::attn_kernel<kExactPartial>", "achieved": sf["s1_flops_attn"] / attn_avg_ms / 1e9,
                     "peak": peak, "unit": "TFLOP/s", "peak_source": "148 SMs x 128 fp32 lanes x 2 flop x 1965 MHz (derived)",
                     "traffic": None}
+        roofline["frac"] = roofline["achieved"] / roofline["peak"]
     else:
-        roofline = {"bound": "tensor", "kernel": "exact-pass attention kernel", "achieved": sf["s1_flops_attn"] / attn_avg_ms / 1e9,
-                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                    "peak_source": f"bf16 cuBLAS sustained, {peaks['source']}", "traffic": None}
-    roofline["frac"] = roofline["achieved"] / roofline["peak"]
+        achieved = sf["s1_flops_attn"] / attn_avg_ms / 1e9
+        roofline = {"bound": "tensor", "kernel": "tc::attn_kernel<false> (Step-1 exact pass over prefix + block keys)", "achieved": achieved,
+                    "peak": peaks["bf16_tflops"] if burst_regime else peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                    "peak_source": f"bf16 cuBLAS {'burst' if burst_regime else 'sustained'}, {peaks['source']}: "
+                                   + ("median SM clock >= 0.95 max and no sw_power_cap sample" if burst_regime else "sw_power_cap sampled or SM clock below 0.95 max"),
+                    "frac_burst": achieved / peaks["bf16_tflops"], "frac_sustained": achieved / peaks["bf16_tflops_sustained"],
+                    "issued_over_useful_flops": float(-(-w.M // 128) * 128) / w.M, "traffic": None}
+        roofline["frac"] = roofline["achieved"] / roofline["peak"]
     roofline["hbm_view"] = {"achieved_gbs": sf["s1_attn_bytes"] / attn_avg_ms / 1e6, "peak_gbs": peaks["hbm_gbs"],
                             "frac_of_measured": sf["s1_attn_bytes"] / attn_avg_ms / 1e6 / peaks["hbm_gbs"],
                             "frac_of_8tbs": sf["s1_attn_bytes"] / attn_avg_ms / 1e6 / 8000.0}
     prof = os.path.join(ROOT, "profiles", "traffic.txt")       # ncu-measured DRAM bytes per launch (see the file's header)
     if os.path.exists(prof):
         for ln in open(prof):
-            f = ln.split()
-            if len(f) == 3 and not ln.startswith("#") and f[0] == ("simt" if args.simt else "default") and f[1] == w.name:
+            f = ln.split(None, 3)
+            if len(f) >= 3 and not ln.startswith("#") and f[0] == ("simt" if args.simt else "default") and f[1] == w.name:
                 roofline["traffic"] = int(f[2])
+                roofline["traffic_source"] = f[3].strip() if len(f) > 3 else "ncu capture, see profiles/traffic.txt"
+    # the stages the benchmark spec names, each against the roof that binds it
+    s1_ms_all = (sum(attn_ms) + sum(comb_ms) + sum(score_ms)) / len(attn_ms)
+    s1_flops = sf["s1_flops_attn"] + sf["s1_flops_score"]
+    tensor_peak = peaks["bf16_tflops"] if burst_regime else peaks["bf16_tflops_sustained"]
+    roofline_stages = {
+        "step1_exact_select": {"bound": "tensor", "achieved": s1_flops / s1_ms_all / 1e9, "peak": tensor_peak, "unit": "TFLOP/s",
+                               "frac": s1_flops / s1_ms_all / 1e9 / tensor_peak, "flops": s1_flops, "ms": s1_ms_all,
+                               "hbm_view": {"algorithmic_bytes": sf["s1_bytes"], "achieved_gbs": sf["s1_bytes"] / s1_ms_all / 1e6,
+                                            "frac_of_measured": sf["s1_bytes"] / s1_ms_all / 1e6 / peaks["hbm_gbs"],
+                                            "frac_of_8tbs": sf["s1_bytes"] / s1_ms_all / 1e6 / 8000.0}}}
+    if stages.get("sparse_step_ms_cold_l2"):
+        sp_ms = stages["sparse_step_ms_cold_l2"]
+        roofline_stages["sparse_reuse_step"] = {"bound": "hbm", "achieved": sf["s3_bytes"] / sp_ms / 1e6, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                                "frac": sf["s3_bytes"] / sp_ms / 1e6 / peaks["hbm_gbs"], "frac_of_8tbs": sf["s3_bytes"] / sp_ms / 1e6 / 8000.0,
+                                                "algorithmic_bytes": sf["s3_bytes"], "ms": sp_ms, "l2": "flushed before each launch"}
 
     cpu_baseline = None
     if not args.no_cpu_baseline:
@@ -455,13 +531,10 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": w.name, "H_q": w.H_q, "H_kv": w.H_kv, "d": w.d, "N": w.N, "B": w.B, "k": w.k, "T": w.T,
-                   "problems": w.P, "cached_tokens": sum(lens), "kv_bytes": sum(lens) * w.H_kv * 512,
-                   "l2_policy": "inputs_larger_than_l2 (KV cache streamed every step evicts L2)",
-                   "parallelism": f"replicas x{world} (independent blocks, no collective)", "kernels": "simt" if args.simt else "default"},
+        "config": config_of(w, lens, world, "simt" if args.simt else "default"),
         "clocks": clocks, "gpu_launches": launches, "dev_status": status,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "roofline": roofline, "cpu_baseline": cpu_baseline, "stages": stages,
+        "roofline": roofline, "roofline_stages": roofline_stages, "cpu_baseline": cpu_baseline, "stages": stages,
     }
     print(json.dumps(line))
     if world > 1:

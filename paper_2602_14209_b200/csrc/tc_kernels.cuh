@@ -140,6 +140,7 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
             for (int dh = 0; dh < 2; ++dh)
                 for (int rb = 0; rb < rows64 / 64; ++rb)
                     tma_load_2d(smem_u32(q_s + dh * (kScoreQBytes / 2) + rb * kBoxBytes), &map_q, bar(Q_FULL), dh * 64, q_row0 + rb * 64);
+            const uint64_t pol_k = l2_policy_evict_first();       // last use of these K lines
             int issued = 0;
             for (int i = 0; i < n_my; ++i) {
                 const int slot = i % kScoreStages, u = i / kScoreStages;
@@ -152,7 +153,7 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                 mbar_arrive_expect_tx(bar(FULL + slot), kTileBytes);
                 for (int kh = 0; kh < 2; ++kh)
                     for (int dh = 0; dh < 2; ++dh)
-                        tma_load_4d(smem_u32(k_s + slot * kTileBytes + dh * kHalfBytes + kh * kBoxBytes), &map_k, bar(FULL + slot), dh * 64, c1[kh], c2[kh], c3[kh]);
+                        tma_load_4d_hint(smem_u32(k_s + slot * kTileBytes + dh * kHalfBytes + kh * kBoxBytes), &map_k, bar(FULL + slot), dh * 64, c1[kh], c2[kh], c3[kh], pol_k);
                 issued = i + 1;
             }
             if (*abort_s) {   // give the copies already in flight a bounded chance to land before the CTA exits
@@ -513,6 +514,10 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
         if (!SPARSE) {
             if (lane == 0) {
                 const int blk_rows_total = kv.P * kv.H_kv * kv.B;
+                // The score pass reads K again right after this pass and its merge: K lines are marked to stay in L2, V lines
+                // (read once) to leave first.  Whether K survives depends on how much of it the launch covers (one layer
+                // of a 32K prefix: 32 MB, it does; a 28-layer 128K batch streams 3.8 GB of K, it does not).
+                const uint64_t pol_k = l2_policy_evict_last(), pol_v = l2_policy_evict_first();
                 int issued = 0;
                 for (int L = 0; L < 2 * n_tiles; ++L) {
                     const int i = L >> 1, is_v = L & 1, slot = slot_of(L);
@@ -533,7 +538,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     for (int kh = 0; kh < 2; ++kh) {
                         if (!blk_chunk) {
                             for (int dh = 0; dh < 2; ++dh)
-                                tma_load_4d(dst + dh * kHalfBytes + kh * kBoxBytes, is_v ? &maps.v : &maps.k, bar(FULL + slot), dh * 64, c1[kh], c2[kh], c3[kh]);
+                                tma_load_4d_hint(dst + dh * kHalfBytes + kh * kBoxBytes, is_v ? &maps.v : &maps.k, bar(FULL + slot), dh * 64, c1[kh], c2[kh], c3[kh], is_v ? pol_v : pol_k);
                         } else {
                             const int row = (i == 0 && kh == 0) ? z * kv.B : blk_rows_total + 64;   // beyond the tensor: zero fill
                             for (int dh = 0; dh < 2; ++dh)

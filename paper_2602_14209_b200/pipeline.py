@@ -48,15 +48,20 @@ class BlockAttention:
         mb.mage_exact_attn(self.kv, q, k_blk, v_blk, self.sm_scale, out, self.workspace, self.status, stream)
         return out
 
+    def select_workspace(self) -> torch.Tensor:
+        """The workspace the select stream's own score pass uses (allocated on first use): it may run while the main
+        stream's Step 1 is using ``self.workspace``."""
+        if getattr(self, "_select_workspace", None) is None:
+            self._select_workspace = self.kv.new_workspace(self.k)
+        return self._select_workspace
+
     def select_scores_async(self, q, workspace: Optional[torch.Tensor] = None, main_stream=None):
         """The paper's two-stream Phase 1: block scores and top-k on the select stream from the queries alone, beside
         whatever the main stream does (its attention, then the FFN).  Uses a workspace of its own (allocated on first use),
         since the main stream's Step 1 may be using ``self.workspace`` at the same time.  Follow with ``join()``."""
         main = torch.cuda.current_stream() if main_stream is None else main_stream
         if workspace is None:
-            if getattr(self, "_select_workspace", None) is None:
-                self._select_workspace = self.kv.new_workspace(self.k)
-            workspace = self._select_workspace
+            workspace = self.select_workspace()
         self._scores_ready.record(main)                   # q is ready on the main stream
         self.select_stream.wait_event(self._scores_ready)
         mb.mage_select_scores(self.kv, q, self.sm_scale, self.scores, workspace, self.status, self.select_stream)
