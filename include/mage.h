@@ -69,6 +69,12 @@ typedef enum {
                                      express, and, in the reuse step on a cache that is not one list of rows with a single
                                      pitch, a cache of more than 2^34 elements. */
 
+#define MAGE_FLAG_TEST_STALL 2    /* test hook for the bounded waits: the exact pass of mage_exact_select / mage_exact_attn /
+                                     mage_select_scores never requests its first key tile, and every wait in that kernel
+                                     gives up after about 1 ms instead of 0.25 s.  The call still returns normally:
+                                     MAGE_DEV_TIMEOUT is set in *dev_status, outputs and scores are undefined, nothing is
+                                     left in flight, and the context stays usable.  Not for production use. */
+
 /*
  * Prefix KV cache "C" of Algorithm 1 for a batch of P problems, read-only.
  *

@@ -18,6 +18,7 @@ _lib = None
 
 MAGE_OK = 0
 FLAG_SIMT_KERNELS = 1
+FLAG_TEST_STALL = 2
 DEV_BAD_INDEX, DEV_BAD_PAGE, DEV_TIMEOUT, DEV_CACHE_FULL = 1, 2, 4, 8
 
 

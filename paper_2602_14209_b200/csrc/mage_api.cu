@@ -204,6 +204,7 @@ static mage_status launch_exact_select(const mage_kv_t *kv, const KvView &view, 
         if (maps_ok && kv->N_max > 0) maps_ok = tc::make_cache_map(&maps.v, kv, kv->v_cache);
         else maps.v = maps.q;
     }
+    maps.test_stall = (kv->flags & MAGE_FLAG_TEST_STALL) ? 1 : 0;
     const bool want_scores = scores && kv->N_max > 0;
     if (maps_ok && want_scores) maps_ok = tc::make_rows_map(&map_q_rows, q, (long long)kv->P * kv->H_q * kv->B) && tc::make_cache_map(&map_k_score, kv, kv->k_cache);
     if (!maps_ok) return MAGE_ERR_UNSUPPORTED;

@@ -59,7 +59,10 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // Every wait in the kernels goes through this: it gives up after ~0.25 s of SM clock (legitimate waits last
 // microseconds), raises the CTA-wide abort flag and the caller's status bit, and returns false.  Once the flag
 // is up, every other wait in the CTA returns false promptly, so all roles fall through to the common exit.
+// abort_flag points at two words of shared memory: [0] the flag, [1] non-zero selects the short limit (~1 ms) that the
+// test hook MAGE_FLAG_TEST_STALL uses to make a wait run out quickly.
 constexpr long long kWaitCycleLimit = 500000000LL;
+constexpr long long kWaitCycleLimitShort = 2000000LL;
 // The polling loop is a function of its own so that the call sites stay short straight-line code (the common case
 // is a phase that is already complete, and the kernels' hot loops should not have to jump over inlined spin loops).
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, unsigned *status) {
@@ -69,7 +72,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
         for (int i = 0; i < 32; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycleLimit) {
+        if (clock64() - t0 > (abort_flag[1] ? kWaitCycleLimitShort : kWaitCycleLimit)) {
             *abort_flag = 1;
             if (status) atomicOr(status, MAGE_DEV_TIMEOUT);
             return false;

@@ -106,7 +106,7 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
     volatile int *abort_s = reinterpret_cast<volatile int *>(tmem_ptr_s + 1);
     // per key tile (ring of 16, far deeper than the producer can run ahead): bit kh set = the 64-key box kh of the tile
     // came from a page id out of range; its keys get score 0
-    volatile int *tile_bad_s = reinterpret_cast<volatile int *>(tmem_ptr_s + 2);
+    volatile int *tile_bad_s = reinterpret_cast<volatile int *>(tmem_ptr_s + 3);
     auto bar = [&](int i) { return smem_u32(bars + i); };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -117,7 +117,8 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
 
     if (tid < 16) tile_bad_s[tid] = 0;
     if (tid == 0) {
-        *abort_s = 0;
+        abort_s[0] = 0;
+        abort_s[1] = 0;                                    // the ordinary wait limit
         mbar_init(bar(Q_FULL), 1);
         for (int s = 0; s < kScoreStages; ++s) { mbar_init(bar(FULL + s), 1); mbar_init(bar(EMPTY + s), 1); }
         for (int b = 0; b < 4; ++b) { mbar_init(bar(T_FULL + b), 1); mbar_init(bar(T_EMPTY + b), 4); }   // one arrival per warp
@@ -381,6 +382,7 @@ __device__ __noinline__ uint32_t sparse_bad_cols(const int *row_tab, const int *
 struct AttnMaps {
     CUtensorMap q, k, v, kb, vb;
     int gather_rows = 0, gather_blk_rows = 0, gather_pitch = 0, lse_only = 0;
+    int test_stall = 0;          // MAGE_FLAG_TEST_STALL: the exact pass never requests its first key tile and waits with the short limit
 };
 
 template <bool SPARSE>
@@ -460,7 +462,8 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid < 8) tile_bad_s[tid] = 0;
     if (tid == 0) {
-        *abort_s = 0;
+        abort_s[0] = 0;
+        abort_s[1] = maps.test_stall;                        // non-zero: waits give up after ~1 ms instead of ~0.25 s
         mbar_init(bar(Q_FULL), 1);
         for (int s = 0; s < kAttnSlots; ++s) { mbar_init(bar(FULL + s), SPARSE ? (maps.gather_rows > 0 ? kSparseProducerWarps : 4) : 1); mbar_init(bar(EMPTY + s), 1); }
         for (int b = 0; b < 2; ++b) {
@@ -522,6 +525,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 for (int L = 0; L < 2 * n_tiles; ++L) {
                     const int i = L >> 1, is_v = L & 1, slot = slot_of(L);
                     if (!mbar_wait(bar(EMPTY + slot), par_of(L) ^ 1, abort_s, status)) break;
+                    if (maps.test_stall) break;                // test hook: K(0) is never requested, so nothing is in flight
                     if (maps.lse_only && is_v) {               // no values in this mode: the slot's phase is completed empty-handed
                         mbar_arrive(bar(FULL + slot));
                         issued = L + 1;
