@@ -116,12 +116,12 @@ def stage_bytes_flops(w, lens):
             "s1_flops_score": s1_flops_score, "s3_bytes": s3_bytes, "s3_flops": s3_flops}
 
 
-def config_of(w, lens, world, kernels):
+def config_of(w, lens, world, kernels, parallelism=None):
     """The `config` object of the JSON line; both arms print the same keys."""
     return {"workload": w.name, "H_q": w.H_q, "H_kv": w.H_kv, "d": w.d, "N": w.N, "B": w.B, "k": w.k, "T": w.T,
             "problems": w.P, "cached_tokens": sum(lens), "kv_bytes": sum(lens) * w.H_kv * 512,
             "l2_policy": "inputs_larger_than_l2 (KV cache streamed every step evicts L2)",
-            "parallelism": f"replicas x{world} (independent blocks, no collective)", "kernels": kernels}
+            "parallelism": parallelism or f"replicas x{world} (independent blocks, no collective)", "kernels": kernels}
 
 
 def spawn_ranks_if_needed(args):
@@ -215,6 +215,9 @@ def main():
     ap.add_argument("--N", type=int, default=None, help="override the prefix length of the workload")
     ap.add_argument("--ragged-min", type=int, default=None,
                     help="override the lower bound of the per-sequence prefix lengths (0 = every sequence has N tokens)")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "kv_head"],
+                    help="N > 1: replicas = every rank runs its own block (weak scaling); kv_head = the ranks split the KV heads of ONE "
+                         "block between them, no collective on the data path (strong scaling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-stage-breakdown", action="store_true")
     ap.add_argument("--bootstrap-only", action="store_true", help="start the ranks, reduce a stand-in time over them and exit (no kernels)")
@@ -257,8 +260,18 @@ def main():
     # weak scaling: every rank runs its own block of the same shape on its own seeded data (independent problems,
     # no data-path collective); rank r draws seed + r.
     import dataclasses
-    w_rank = dataclasses.replace(w, seed=w.seed + rank)
-    batch = W.make_batch(w_rank, device=dev)
+    kv_head_sharded = args.shard == "kv_head" and world > 1
+    w_full = w
+    if kv_head_sharded:
+        # strong scaling: ONE block; rank r owns KV heads [r*H_kv/W, (r+1)*H_kv/W) of every layer and their G query heads.
+        # Every stage is independent per KV head (Eq. 2 / Eq. 4 sum only inside group(h)): no data-path collective.
+        if w.page_size:
+            raise SystemExit("--shard kv_head is implemented for contiguous caches")
+        batch = W.make_batch(w, device=dev)                                   # same seed on every rank: the same block
+        w, batch = W.shard_batch_by_kv_head(batch, w, world, rank)             # strided views of the cache, no copy
+    else:
+        w_rank = dataclasses.replace(w, seed=w.seed + rank)
+        batch = W.make_batch(w_rank, device=dev)
     lens = [int(x) for x in batch["seq_lens"].tolist()]
     flags = mb.FLAG_SIMT_KERNELS if args.simt else 0
     if w.page_size:
@@ -346,8 +359,11 @@ def main():
         dist.all_reduce(lt)
         launches = int(lt[0])
     ms_per_step = ms_total / args.steps
-    value = ms_per_step / world                 # ms per block over the whole job: each of the N ranks finishes one block per step
-    e2e_value = e2e_ms_total / e2e_steps / world
+    if kv_head_sharded:
+        value, e2e_value = ms_per_step, e2e_ms_total / e2e_steps          # one block per step for the whole job
+    else:
+        value = ms_per_step / world             # ms per block over the whole job: each of the N ranks finishes one block per step
+        e2e_value = e2e_ms_total / e2e_steps / world
 
     # ---- per-stage numbers (rank 0, outside the headline region): sparse step cold/warm, top-k alone -------------
     stages = {}
@@ -529,9 +545,10 @@ def main():
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "strong" if kv_head_sharded else "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": config_of(w, lens, world, "simt" if args.simt else "default"),
+        "config": config_of(w_full, lens, world, "simt" if args.simt else "default",
+                            f"kv_head x{world} (each rank owns H_kv/{world} KV heads of every layer; no collective)" if kv_head_sharded else None),
         "clocks": clocks, "gpu_launches": launches, "dev_status": status,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "roofline": roofline, "roofline_stages": roofline_stages, "cpu_baseline": cpu_baseline, "stages": stages,

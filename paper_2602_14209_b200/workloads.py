@@ -249,3 +249,21 @@ def shard_by_kv_head(H_q: int, H_kv: int, world_size: int, rank: int):
 def shard_problems(P: int, world_size: int, rank: int) -> List[int]:
     """Round-robin split of independent problems (layers / sequences) across ranks."""
     return list(range(rank, P, world_size))
+
+
+def shard_batch_by_kv_head(batch: dict, w: Workload, world_size: int, rank: int):
+    """The slice of a `make_batch` result that rank `rank` of `world_size` owns under KV-head sharding.
+
+    Returns (local_workload, local_batch).  The cache tensors are strided VIEWS of the full ones (head stride and problem
+    stride unchanged: the library takes them as they are); queries, block keys and block values are small and are
+    copied into the contiguous [.., H_local, B, d] layout the library expects.  Nothing here needs another rank's data.
+    """
+    hs, qs = shard_by_kv_head(w.H_q, w.H_kv, world_size, rank)
+    local = dataclasses.replace(w, name=f"{w.name}[kv_heads {hs.start}:{hs.stop}]", H_q=qs.stop - qs.start, H_kv=hs.stop - hs.start)
+    out = dict(batch)
+    out["kc"], out["vc"] = batch["kc"][:, hs], batch["vc"][:, hs]
+    out["q"] = batch["q"][:, :, qs].contiguous()
+    out["kb"], out["vb"] = batch["kb"][:, :, hs].contiguous(), batch["vb"][:, :, hs].contiguous()
+    out["heavy"] = [h[hs] for h in batch["heavy"]]
+    return local, out
+
