@@ -411,6 +411,23 @@ def main():
             "sparse_step_tflops_cold": sf["s3_flops"] / sp_cold / 1e9,
             "hbm_roofline_ms_block_at_8tbs": (sf["s1_bytes"] + (T - 1) * sf["s3_bytes"]) / 8e9,
         }
+        # The paper's comparison system on the same inputs: a Quest-style page estimator (16-token pages) re-estimated at
+        # every step = page scores + page top-k + index expansion, then the same reuse-step kernel on its index set.
+        if w.k % mb.QUEST_PAGE == 0 and kv.N_max >= mb.QUEST_PAGE:
+            n_pg = (kv.N_max + mb.QUEST_PAGE - 1) // mb.QUEST_PAGE
+            pmin = torch.empty(kv.P, kv.H_kv, n_pg, kv.d, dtype=torch.bfloat16, device=dev)
+            pmax = torch.empty_like(pmin)
+            psc = torch.empty(kv.P, kv.H_kv, n_pg, dtype=torch.float32, device=dev)
+            q_idx, q_keff, q_ws = torch.empty_like(ba.indices), torch.empty_like(ba.k_eff), mb.quest_workspace(kv, w.k)
+            qb = lambda: mb.mage_quest_build(kv, pmin, pmax, ba.status)
+            qs = lambda: mb.mage_quest_select(kv, q_d[1], pmin, pmax, w.k, psc, q_idx, q_keff, q_ws)
+            qb(); qs(); torch.cuda.synchronize()
+            qsp = lambda: mb.mage_sparse_block_attn(kv, q_d[1], kb_d[1], vb_d[1], q_idx, q_keff, w.k, ba.sm_scale, outs[1], ba.workspace, ba.status)
+            stages["quest_build_ms"] = timed(qb, True, 5)
+            stages["quest_select_ms_cold_l2"] = timed(qs, True, 5)
+            stages["quest_step_ms_cold_l2"] = stages["quest_select_ms_cold_l2"] + timed(qsp, True, 5)
+            stages["quest_summary_bytes"] = 2 * pmin.numel() * 2
+            del pmin, pmax, psc
         del flush
         # The same block issued layer by layer, as a model would (config 3 "timed back-to-back"): one exact_select, one
         # top-k (select stream) and T-1 sparse launches per layer; plain launches, and replayed from a CUDA graph.

@@ -243,6 +243,31 @@ mage_status mage_select_scores(const mage_kv_t *kv, const void *q, float sm_scal
 mage_status mage_exact_select_static(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk,
                                      float sm_scale, void *out, float *scores, uint32_t *dev_status, void *stream);
 
+/*
+ * Quest-style page estimator in its per-block form: the paper's comparison system on the same inputs, not a part of
+ * MAGE (Section 2.2: pages of p tokens summarised by per-channel max / min keys, page score = the sign-aware upper
+ * bound sum_c max(q_c Kmax_c, q_c Kmin_c) on q.k; Section 3.1, Eq. 2 with that estimate as s: the mean over the
+ * block's G*B queries; Section 5, Setup: p = 16, re-estimated at every denoising step).
+ *
+ * mage_quest_build summarises the whole pages of every prefix (positions [0, 16*floor(N_p/16)); a ragged tail of
+ * fewer than 16 tokens is never a candidate):
+ *   page_min, page_max  [P][H_kv][ceil(N_max/16)][d] bf16, device, written for whole pages only
+ * mage_quest_select scores the pages against the current queries, takes the k/16 best pages per KV head (exact,
+ * ties to the smaller page) and writes their tokens as an index set that mage_sparse_block_attn accepts:
+ *   q            [P][H_q][B][d] bf16
+ *   k            a multiple of 16
+ *   page_scores  [P][H_kv][ceil(N_max/16)] fp32, written for whole pages
+ *   indices      [P][H_kv][k] int32 ascending, -1 padded;  k_eff [P] int32 = 16 * min(k/16, floor(N_p/16))
+ *   workspace    device, 256-byte aligned, at least mage_quest_workspace_bytes(kv, k)
+ * Cache page sizes must be multiples of 16 (or 0).  Errors as the other calls; nothing is launched unless MAGE_OK.
+ */
+#define MAGE_QUEST_PAGE 16
+size_t mage_quest_workspace_bytes(const mage_kv_t *kv, int32_t k);
+mage_status mage_quest_build(const mage_kv_t *kv, void *page_min, void *page_max, uint32_t *dev_status, void *stream);
+mage_status mage_quest_select(const mage_kv_t *kv, const void *q, const void *page_min, const void *page_max, int32_t k,
+                              float *page_scores, int32_t *indices, int32_t *k_eff, void *workspace, size_t workspace_bytes,
+                              void *stream);
+
 /* Static, human-readable name of a status code. */
 const char *mage_status_string(mage_status s);
 

@@ -5,4 +5,4 @@ legs of ``bench.py`` may import this package.  It shares no code with the CUDA
 library and never imports it.
 """
 from .oracle import (build, exact_block_attn, block_score, topk, sparse_block_attn, recall,  # noqa: F401
-                     num_threads, run_block)
+                     num_threads, run_block, quest_page_summaries, quest_page_scores, quest_select)

@@ -113,3 +113,50 @@ def run_block(q_steps, Kc, Vc, kb_steps, vb_steps, k, scale=None):
     Os = [sparse_block_attn(q_steps[t], Kc, Vc, kb_steps[t], vb_steps[t], idx, k_eff, scale)
           for t in range(1, len(q_steps))]
     return {"O_exact": O1, "score": sc, "idx": idx, "k_eff": k_eff, "O_sparse": Os}
+
+
+# ---------------------------------------------------------------------------------------------------------------------
+# Quest-style page estimator in its per-block form (the paper's comparison system; Section 2.2 for the estimator,
+# Section 3.1 / Eq. 2 for the per-block mean, Section 5 "Setup" for page size 16).  Plain NumPy in float64, written as
+# the definitions read: per-channel extremes of each page, the sign-aware bound evaluated per query row with the max
+# inside the sum over channels, then the mean over the block's G*B rows.
+# ---------------------------------------------------------------------------------------------------------------------
+def quest_page_summaries(Kc, page=16):
+    """Per-channel min / max keys of each whole page (Section 2.2).  Kc [H_kv,N,d] -> (kmin, kmax) [H_kv, N // page, d]."""
+    Kc = np.asarray(Kc, dtype=np.float64)
+    H_kv, N, d = Kc.shape
+    n_pages = N // page
+    blocks = Kc[:, : n_pages * page].reshape(H_kv, n_pages, page, d)
+    return blocks.min(axis=2), blocks.max(axis=2)
+
+
+def quest_page_scores(Q, kmin, kmax):
+    """Per-block page score: 1/(G B) * sum over g in group(h), q in block of sum_c max(Q[g,q,c] Kmax[c], Q[g,q,c] Kmin[c])
+    (Section 2.2 for the inner bound; Eq. 2's per-block form with that bound as s).  Q [H_q,B,d] -> [H_kv, n_pages]."""
+    Q = np.asarray(Q, dtype=np.float64)
+    H_q, B, d = Q.shape
+    H_kv, n_pages, _ = kmin.shape
+    G = H_q // H_kv
+    score = np.zeros((H_kv, n_pages))
+    for h in range(H_kv):
+        for g in range(h * G, (h + 1) * G):
+            for qi in range(B):
+                qv = Q[g, qi]                                             # [d]
+                score[h] += np.maximum(qv[None, :] * kmax[h], qv[None, :] * kmin[h]).sum(axis=1)
+    return score / (G * B)
+
+
+def quest_select(Q, Kc, k, page=16):
+    """The k/page best pages per KV head and their tokens.  Returns (idx [H_kv,k] int32 ascending, -1 padded; k_eff; page scores)."""
+    kmin, kmax = quest_page_summaries(Kc, page)
+    sc = quest_page_scores(Q, kmin, kmax)
+    H_kv, n_pages = sc.shape
+    k_pages = k // page
+    idx = np.full((H_kv, k), -1, dtype=np.int32)
+    n_sel = min(k_pages, n_pages)
+    if n_pages > 0:
+        pages, n_sel = topk(sc, k_pages)
+        for h in range(H_kv):
+            idx[h, : n_sel * page] = (pages[h, :n_sel, None].astype(np.int64) * page + np.arange(page)[None, :]).reshape(-1)
+    return idx, n_sel * page, sc
+

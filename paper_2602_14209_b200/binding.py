@@ -39,7 +39,7 @@ class mage_kv_t(ctypes.Structure):
     ]
 
 
-EXPORTS = ("mage_append_block", "mage_workspace_bytes", "mage_exact_select", "mage_exact_select_events", "mage_exact_select_static", "mage_exact_attn", "mage_select_scores", "mage_topk", "mage_sparse_block_attn",
+EXPORTS = ("mage_quest_workspace_bytes", "mage_quest_build", "mage_quest_select", "mage_append_block", "mage_workspace_bytes", "mage_exact_select", "mage_exact_select_events", "mage_exact_select_static", "mage_exact_attn", "mage_select_scores", "mage_topk", "mage_sparse_block_attn",
            "mage_status_string", "mage_launch_count")
 
 
@@ -70,6 +70,12 @@ def load():
     lib.mage_sparse_block_attn.argtypes = [ctypes.POINTER(mage_kv_t), vp, vp, vp, vp, vp, i32, ctypes.c_float, vp, vp, ctypes.c_size_t, vp, vp]
     lib.mage_append_block.restype = ctypes.c_int
     lib.mage_append_block.argtypes = [ctypes.POINTER(mage_kv_t), vp, vp, vp, vp, vp]
+    lib.mage_quest_workspace_bytes.restype = ctypes.c_size_t
+    lib.mage_quest_workspace_bytes.argtypes = [ctypes.POINTER(mage_kv_t), i32]
+    lib.mage_quest_build.restype = ctypes.c_int
+    lib.mage_quest_build.argtypes = [ctypes.POINTER(mage_kv_t), vp, vp, vp, vp]
+    lib.mage_quest_select.restype = ctypes.c_int
+    lib.mage_quest_select.argtypes = [ctypes.POINTER(mage_kv_t), vp, vp, vp, i32, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.mage_status_string.restype = ctypes.c_char_p
     lib.mage_status_string.argtypes = [ctypes.c_int]
     lib.mage_launch_count.restype = u64
@@ -221,3 +227,29 @@ def mage_append_block(kv: KVCache, k_blk, v_blk, seq_lens, dev_status=None, stre
     rc = load().mage_append_block(ctypes.byref(kv.c), _ptr(k_blk), _ptr(v_blk), _ptr(seq_lens), _ptr(dev_status), _stream(stream))
     if rc != MAGE_OK:
         raise MageError(rc, "mage_append_block")
+
+
+QUEST_PAGE = 16
+
+
+def mage_quest_build(kv: KVCache, page_min, page_max, dev_status=None, stream=None):
+    """Quest-style page summaries (per-channel min / max of each whole 16-token page of the prefix; see mage.h)."""
+    rc = load().mage_quest_build(ctypes.byref(kv.c), _ptr(page_min), _ptr(page_max), _ptr(dev_status), _stream(stream))
+    if rc != MAGE_OK:
+        raise MageError(rc, "mage_quest_build")
+
+
+def mage_quest_select(kv: KVCache, q, page_min, page_max, k: int, page_scores, indices, k_eff, workspace, stream=None):
+    """Per-block Quest-style selection: page scores, the k/16 best pages, their tokens as an index set (see mage.h)."""
+    rc = load().mage_quest_select(ctypes.byref(kv.c), _ptr(q), _ptr(page_min), _ptr(page_max), int(k), _ptr(page_scores), _ptr(indices),
+                                  _ptr(k_eff), _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
+    if rc != MAGE_OK:
+        raise MageError(rc, "mage_quest_select")
+
+
+def quest_workspace(kv: KVCache, k: int) -> torch.Tensor:
+    n = int(load().mage_quest_workspace_bytes(ctypes.byref(kv.c), int(k)))
+    if n == 0:
+        raise MageError(-1, "mage_quest_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=kv.device)
+

@@ -6,6 +6,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "quest.cuh"
 #include "simt_kernels.cuh"
 #include "tc_host.cuh"
 #include "topk.cuh"
@@ -424,6 +425,51 @@ mage_status mage_exact_select_static(const mage_kv_t *kv, const void *q, const v
     }
     return mage_exact_select_events(kv, q, k_blk, v_blk, sm_scale, out, scores, scratch, (size_t)MAGE_STATIC_SCRATCH_BYTES,
                                     dev_status, stream, nullptr);
+}
+
+size_t mage_quest_workspace_bytes(const mage_kv_t *kv, int32_t k) {
+    if (!valid_kv(kv, nullptr) || k < MAGE_QUEST_PAGE || k % MAGE_QUEST_PAGE) return 0;
+    // page counts [P], selected-page counts [P], selected pages [P][H_kv][k/16]
+    return align_up((size_t)kv->P * 2 * sizeof(int), 256) + align_up((size_t)kv->P * kv->H_kv * (k / MAGE_QUEST_PAGE) * sizeof(int), 256);
+}
+
+mage_status mage_quest_build(const mage_kv_t *kv, void *page_min, void *page_max, uint32_t *dev_status, void *stream) {
+    mage_status why = MAGE_OK;
+    if (!valid_kv(kv, &why)) return why;
+    if (kv->page_size % MAGE_QUEST_PAGE) return MAGE_ERR_UNSUPPORTED;
+    if (kv->N_max < MAGE_QUEST_PAGE) return MAGE_OK;              // no whole page anywhere
+    if (!page_min || !page_max) return MAGE_ERR_INVALID_ARG;
+    const KvView view = make_view(kv);
+    const int n_pages_max = (kv->N_max + MAGE_QUEST_PAGE - 1) / MAGE_QUEST_PAGE;
+    const long long warps = (long long)kv->P * kv->H_kv * n_pages_max;
+    quest::build_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, static_cast<cudaStream_t>(stream)>>>(view, n_pages_max, static_cast<__nv_bfloat16 *>(page_min),
+                                                                                                  static_cast<__nv_bfloat16 *>(page_max), dev_status);
+    return launch_check();
+}
+
+mage_status mage_quest_select(const mage_kv_t *kv, const void *q, const void *page_min, const void *page_max, int32_t k,
+                              float *page_scores, int32_t *indices, int32_t *k_eff, void *workspace, size_t workspace_bytes,
+                              void *stream) {
+    mage_status why = MAGE_OK;
+    if (!valid_kv(kv, &why)) return why;
+    if (k < MAGE_QUEST_PAGE || k % MAGE_QUEST_PAGE || !q || !indices || !k_eff || !workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return MAGE_ERR_INVALID_ARG;
+    if (kv->page_size % MAGE_QUEST_PAGE) return MAGE_ERR_UNSUPPORTED;
+    if (workspace_bytes < mage_quest_workspace_bytes(kv, k)) return MAGE_ERR_WORKSPACE;
+    const int n_pages_max = (kv->N_max + MAGE_QUEST_PAGE - 1) / MAGE_QUEST_PAGE;
+    if (n_pages_max > 0 && (!page_min || !page_max || !page_scores)) return MAGE_ERR_INVALID_ARG;
+    const KvView view = make_view(kv);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int heads = kv->P * kv->H_kv, k_pages = k / MAGE_QUEST_PAGE;
+    int *page_counts = static_cast<int *>(workspace), *pages_sel = page_counts + kv->P;
+    int *page_idx = reinterpret_cast<int *>(static_cast<char *>(workspace) + align_up((size_t)kv->P * 2 * sizeof(int), 256));
+    quest::score_kernel<<<dim3(std::max(1, (n_pages_max + quest::kPagesPerCta - 1) / quest::kPagesPerCta), heads), 256, 0, st>>>(
+        view, n_pages_max, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(page_min),
+        static_cast<const __nv_bfloat16 *>(page_max), page_scores, page_counts);
+    if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    topk_kernel<<<heads, kTopkThreads, 0, st>>>(page_scores, page_counts, kv->H_kv, n_pages_max, k_pages, page_idx, pages_sel);
+    if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    quest::expand_kernel<<<heads, 256, 0, st>>>(kv->H_kv, k, page_idx, pages_sel, indices, k_eff);
+    return launch_check();
 }
 
 const char *mage_status_string(mage_status s) {

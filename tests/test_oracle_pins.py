@@ -211,3 +211,72 @@ def test_recall_known_answers(oracle_mod):
     b = np.array([[40, 50, 60, 70], [1, 2, 3, 9]], dtype=np.int32)
     assert oracle_mod.recall(a, b, 4).tolist() == [0.25, 0.75]
 
+
+# ---- Quest-style page estimator (comparison system): pins for the oracle's restatement -----------------------------
+def _quest_inputs(seed, H_q=4, H_kv=2, B=3, N=70, d=8):
+    rng = np.random.default_rng(seed)
+    from helpers import bf16_exact
+    return bf16_exact(rng, (H_q, B, d)), bf16_exact(rng, (H_kv, N, d))
+
+
+def test_quest_page_score_brute_force_loops(oracle_mod):
+    """Pure-Python loops over pages, tokens, channels, rows on a tiny case (including a ragged tail that is no page)."""
+    Q, Kc = _quest_inputs(1)
+    H_q, B, d = Q.shape
+    H_kv, N, _ = Kc.shape
+    G, page = H_q // H_kv, 16
+    kmin, kmax = oracle_mod.quest_page_summaries(Kc, page)
+    sc = oracle_mod.quest_page_scores(Q, kmin, kmax)
+    assert kmin.shape == (H_kv, N // page, d) and sc.shape == (H_kv, N // page)
+    for h in range(H_kv):
+        for pg in range(N // page):
+            total = 0.0
+            for g in range(h * G, (h + 1) * G):
+                for qi in range(B):
+                    for c in range(d):
+                        lo = min(float(Kc[h, pg * page + t, c]) for t in range(page))
+                        hi = max(float(Kc[h, pg * page + t, c]) for t in range(page))
+                        total += max(float(Q[g, qi, c]) * hi, float(Q[g, qi, c]) * lo)
+            np.testing.assert_allclose(sc[h, pg], total / (G * B), rtol=1e-12, atol=1e-12)
+
+
+def test_quest_bound_dominates_every_key_of_its_page(oracle_mod):
+    """The defining property (Section 2.2): per query, the page bound is an upper bound on q.k for every key of the page,
+    so the per-block page score is at least the mean over rows of the page's best exact logit."""
+    Q, Kc = _quest_inputs(2, H_q=6, H_kv=2, B=4, N=96, d=16)
+    kmin, kmax = oracle_mod.quest_page_summaries(Kc)
+    sc = oracle_mod.quest_page_scores(Q, kmin, kmax)
+    G = 3
+    for h in range(2):
+        rows = Q[h * G:(h + 1) * G].reshape(-1, 16).astype(np.float64)
+        logits = rows @ Kc[h].astype(np.float64).T                        # [M, N]
+        best = logits.reshape(rows.shape[0], 6, 16).max(axis=2)            # per row and page
+        assert (sc[h] >= best.mean(axis=0) - 1e-12).all()
+        # and a transposed or sign-flipped bound would violate it somewhere: the bound is tight for single-key pages
+    kmin1, kmax1 = oracle_mod.quest_page_summaries(Kc, page=1)
+    sc1 = oracle_mod.quest_page_scores(Q, kmin1, kmax1)
+    for h in range(2):
+        rows = Q[h * G:(h + 1) * G].reshape(-1, 16).astype(np.float64)
+        np.testing.assert_allclose(sc1[h], (rows @ Kc[h].astype(np.float64).T).mean(axis=0), rtol=1e-12, atol=1e-12)
+
+
+def test_quest_closed_forms_and_selection(oracle_mod):
+    """All keys of a page equal -> the bound is the exact logit; positive queries -> only Kmax matters; the selected
+    tokens are whole pages, ascending, and the ragged tail is never selected."""
+    rng = np.random.default_rng(3)
+    from helpers import bf16_exact
+    Q = np.abs(bf16_exact(rng, (2, 2, 8))) + 0.5
+    Kc = bf16_exact(rng, (1, 52, 8))
+    Kc[0, 16:32] = Kc[0, 16]                                               # page 1: sixteen copies of one key
+    kmin, kmax = oracle_mod.quest_page_summaries(Kc)
+    sc = oracle_mod.quest_page_scores(Q, kmin, kmax)
+    rows = Q.reshape(-1, 8).astype(np.float64)
+    np.testing.assert_allclose(sc[0, 1], (rows @ Kc[0, 16].astype(np.float64)).mean(), rtol=1e-12)
+    np.testing.assert_allclose(sc[0], (rows @ kmax[0].T).mean(axis=0), rtol=1e-12)      # q > 0: the max keys alone
+    idx, k_eff, _ = oracle_mod.quest_select(Q, Kc, 32)
+    assert k_eff == 32 and (np.diff(idx[0]) > 0).all() and idx.max() < 48               # positions 48..51 are no page
+    best2 = np.sort(np.argsort(-sc[0], kind="stable")[:2])
+    assert idx[0].tolist() == [int(p) * 16 + t for p in best2 for t in range(16)]
+    idx, k_eff, _ = oracle_mod.quest_select(Q, Kc, 64)                                   # more pages asked than exist
+    assert k_eff == 48 and (idx[0, 48:] == -1).all() and idx[0, :48].tolist() == list(range(48))
+
