@@ -411,6 +411,21 @@ def main():
             "sparse_step_tflops_cold": sf["s3_flops"] / sp_cold / 1e9,
             "hbm_roofline_ms_block_at_8tbs": (sf["s1_bytes"] + (T - 1) * sf["s3_bytes"]) / 8e9,
         }
+        # Step 1 + selection with the score pass restricted to the tiles that can hold a selected key, beside the plain pair
+        # (exact_select + top-k, same stream).  On flat attention nothing can be pruned and the call pays its bookkeeping.
+        pw = mb.pruned_workspace(kv, w.k)
+        p_idx, p_keff, p_tiles = torch.empty_like(ba.indices), torch.empty_like(ba.k_eff), torch.zeros(kv.P, kv.H_kv, dtype=torch.int32, device=dev)
+        pruned = lambda: mb.mage_exact_select_pruned(kv, q_d[0], kb_d[0], vb_d[0], ba.sm_scale, w.k, outs[0], ba.scores, p_idx, p_keff, pw,
+                                                     tiles_scored=p_tiles, dev_status=ba.status)
+        plain = lambda: (ba.exact_select(q_d[0], kb_d[0], vb_d[0], outs[0]), tk())
+        plain(); torch.cuda.synchronize()
+        idx_plain = ba.indices.clone()
+        pruned(); torch.cuda.synchronize()
+        tiles_all = sum((n + 127) // 128 for n in lens) * w.H_kv
+        stages["pruned_select_ms"], stages["plain_select_ms_same_stream"] = timed(pruned, False, 5), timed(plain, False, 5)
+        stages["pruned_tiles_scored_frac"] = float(p_tiles.sum().item()) / max(1, tiles_all)
+        stages["pruned_same_index_sets"] = bool(torch.equal(p_idx, idx_plain))
+        del pw
         # The paper's comparison system on the same inputs: a Quest-style page estimator (16-token pages) re-estimated at
         # every step = page scores + page top-k + index expansion, then the same reuse-step kernel on its index set.
         if w.k % mb.QUEST_PAGE == 0 and kv.N_max >= mb.QUEST_PAGE:

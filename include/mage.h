@@ -244,6 +244,29 @@ mage_status mage_exact_select_static(const mage_kv_t *kv, const void *q, const v
                                      float sm_scale, void *out, float *scores, uint32_t *dev_status, void *stream);
 
 /*
+ * Step 1 and the selection in one call, scoring only where a selected key can be (Algorithm 1, Phase 1: main-stream
+ * "Attn(Q, K, V, C)", select-stream "alpha", "S <- Top-k(alpha)"; Eq. 4).  The result -- out, indices, k_eff -- is that
+ * of mage_exact_select followed by mage_topk; what differs is the work: the exact pass records, per 128-key tile and
+ * query row, the probability mass the row puts on the tile; a key's score is at most its tile's mass averaged over
+ * rows; tiles whose mass is below the k-th largest exact score found among the heaviest tiles cannot hold a selected key
+ * and are not scored (their entries of `scores` are written as 0).  On flat attention every tile is scored, as in
+ * mage_exact_select; on concentrated attention the second pass over K shrinks to the tiles that matter.
+ *
+ *   k            budget, as in mage_topk
+ *   dense_above  when more than this fraction (0..1) of a head's remaining tiles would be scored anyway, all of them are
+ *   scores       [P][H_kv][N_max] fp32: exact (Eq. 4) in scored tiles, 0 elsewhere below N_p; untouched from N_p on
+ *   indices, k_eff  as mage_topk writes them
+ *   tiles_scored [P][H_kv] int32, optional (may be NULL): key tiles of each head that went through the score pass
+ *   workspace    device, 256-byte aligned, at least mage_pruned_workspace_bytes(kv, k)
+ * Runs on `stream` only.  Not available with MAGE_FLAG_SIMT_KERNELS (MAGE_ERR_UNSUPPORTED).
+ */
+size_t mage_pruned_workspace_bytes(const mage_kv_t *kv, int32_t k);
+mage_status mage_exact_select_pruned(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk, float sm_scale,
+                                     int32_t k, float dense_above, void *out, float *scores, int32_t *indices, int32_t *k_eff,
+                                     int32_t *tiles_scored, void *workspace, size_t workspace_bytes, uint32_t *dev_status,
+                                     void *stream);
+
+/*
  * Quest-style page estimator in its per-block form: the paper's comparison system on the same inputs, not a part of
  * MAGE (Section 2.2: pages of p tokens summarised by per-channel max / min keys, page score = the sign-aware upper
  * bound sum_c max(q_c Kmax_c, q_c Kmin_c) on q.k; Section 3.1, Eq. 2 with that estimate as s: the mean over the

@@ -39,7 +39,7 @@ class mage_kv_t(ctypes.Structure):
     ]
 
 
-EXPORTS = ("mage_quest_workspace_bytes", "mage_quest_build", "mage_quest_select", "mage_append_block", "mage_workspace_bytes", "mage_exact_select", "mage_exact_select_events", "mage_exact_select_static", "mage_exact_attn", "mage_select_scores", "mage_topk", "mage_sparse_block_attn",
+EXPORTS = ("mage_pruned_workspace_bytes", "mage_exact_select_pruned", "mage_quest_workspace_bytes", "mage_quest_build", "mage_quest_select", "mage_append_block", "mage_workspace_bytes", "mage_exact_select", "mage_exact_select_events", "mage_exact_select_static", "mage_exact_attn", "mage_select_scores", "mage_topk", "mage_sparse_block_attn",
            "mage_status_string", "mage_launch_count")
 
 
@@ -70,6 +70,11 @@ def load():
     lib.mage_sparse_block_attn.argtypes = [ctypes.POINTER(mage_kv_t), vp, vp, vp, vp, vp, i32, ctypes.c_float, vp, vp, ctypes.c_size_t, vp, vp]
     lib.mage_append_block.restype = ctypes.c_int
     lib.mage_append_block.argtypes = [ctypes.POINTER(mage_kv_t), vp, vp, vp, vp, vp]
+    lib.mage_pruned_workspace_bytes.restype = ctypes.c_size_t
+    lib.mage_pruned_workspace_bytes.argtypes = [ctypes.POINTER(mage_kv_t), i32]
+    lib.mage_exact_select_pruned.restype = ctypes.c_int
+    lib.mage_exact_select_pruned.argtypes = [ctypes.POINTER(mage_kv_t), vp, vp, vp, ctypes.c_float, i32, ctypes.c_float, vp, vp, vp, vp, vp, vp,
+                                             ctypes.c_size_t, vp, vp]
     lib.mage_quest_workspace_bytes.restype = ctypes.c_size_t
     lib.mage_quest_workspace_bytes.argtypes = [ctypes.POINTER(mage_kv_t), i32]
     lib.mage_quest_build.restype = ctypes.c_int
@@ -252,4 +257,21 @@ def quest_workspace(kv: KVCache, k: int) -> torch.Tensor:
     if n == 0:
         raise MageError(-1, "mage_quest_workspace_bytes")
     return torch.empty(n, dtype=torch.uint8, device=kv.device)
+
+
+def pruned_workspace(kv: KVCache, k: int) -> torch.Tensor:
+    n = int(load().mage_pruned_workspace_bytes(ctypes.byref(kv.c), int(k)))
+    if n == 0:
+        raise MageError(-1, "mage_pruned_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=kv.device)
+
+
+def mage_exact_select_pruned(kv: KVCache, q, k_blk, v_blk, sm_scale: float, k: int, out, scores, indices, k_eff, workspace,
+                             tiles_scored=None, dense_above: float = 0.5, dev_status=None, stream=None):
+    """Step 1 + selection with the score pass restricted to the key tiles that can hold a selected key (see mage.h)."""
+    rc = load().mage_exact_select_pruned(ctypes.byref(kv.c), _ptr(q), _ptr(k_blk), _ptr(v_blk), float(sm_scale), int(k), float(dense_above),
+                                         _ptr(out), _ptr(scores), _ptr(indices), _ptr(k_eff), _ptr(tiles_scored), _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream(stream))
+    if rc != MAGE_OK:
+        raise MageError(rc, "mage_exact_select_pruned")
 

@@ -6,6 +6,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "prune.cuh"
 #include "quest.cuh"
 #include "simt_kernels.cuh"
 #include "tc_host.cuh"
@@ -157,6 +158,19 @@ static mage_status tc_supported(const mage_kv_t *kv) {
     return MAGE_OK;
 }
 
+// The block-score pass (Eq. 4) over all key tiles, or over the tiles of `list`: grid_x CTAs of tiles_per_cta tiles per head.
+static mage_status launch_score_pass(const KvView &view, const Plan &plan, const CUtensorMap &map_q_rows, const CUtensorMap &map_k,
+                                     int grid_x, int tiles_per_cta, float scale_log2, const float *ws, float *scores,
+                                     unsigned *dev_status, cudaStream_t st, const tc::ScoreTileList &list) {
+    dim3 sgrid(grid_x, view.P * view.H_kv, 1);
+    for (int r0 = 0; r0 < view.M; r0 += 256) {
+        launch_pdl(tc::score_kernel, sgrid, dim3(tc::kScoreThreads), tc::kScoreSmemBytes, st, map_q_rows, map_k, view, plan, r0, std::min(256, view.M - r0),
+                   tiles_per_cta, scale_log2, ws, scores, (int)(r0 > 0), dev_status, list);
+        if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    }
+    return MAGE_OK;
+}
+
 // Step 1 (Algorithm 1, Phase 1): the exact pass over prefix + block keys, the merge of its per-chunk partial results and
 // the block-score pass.  scores_only: the select stream's own computation (Algorithm 1: A = softmax(Q K^T / sqrt d) over
 // the prefix, then the mean over the block's rows) without the attention output: pass A keeps only the rows' maxima and
@@ -164,7 +178,7 @@ static mage_status tc_supported(const mage_kv_t *kv) {
 static mage_status launch_exact_select(const mage_kv_t *kv, const KvView &view, const Plan &plan, const __nv_bfloat16 *q,
                                        const __nv_bfloat16 *k_blk, const __nv_bfloat16 *v_blk, float sm_scale,
                                        __nv_bfloat16 *out, float *scores, float *ws, unsigned *dev_status, cudaStream_t st,
-                                       cudaEvent_t *ev, bool scores_only = false) {
+                                       cudaEvent_t *ev, bool scores_only = false, float2 *rowsum = nullptr, int rowsum_tiles = 0) {
     const float scale_log2 = sm_scale * kLog2e;
     const int heads = kv->P * kv->H_kv, rows_total = heads * view.M;
     const int n_items = plan.n_chunks + (scores_only ? 0 : 1);
@@ -206,6 +220,8 @@ static mage_status launch_exact_select(const mage_kv_t *kv, const KvView &view, 
         else maps.v = maps.q;
     }
     maps.test_stall = (kv->flags & MAGE_FLAG_TEST_STALL) ? 1 : 0;
+    maps.rowsum = rowsum;
+    maps.rowsum_tiles = rowsum_tiles;
     const bool want_scores = scores && kv->N_max > 0;
     if (maps_ok && want_scores) maps_ok = tc::make_rows_map(&map_q_rows, q, (long long)kv->P * kv->H_q * kv->B) && tc::make_cache_map(&map_k_score, kv, kv->k_cache);
     if (!maps_ok) return MAGE_ERR_UNSUPPORTED;
@@ -223,12 +239,8 @@ static mage_status launch_exact_select(const mage_kv_t *kv, const KvView &view, 
     if (want_scores) {
         const int tpc = tc::tiles_per_cta_for(heads, kv->N_max, kv->page_size != 0);
         const int tiles_head = (kv->N_max + tc::kTile - 1) / tc::kTile;
-        dim3 sgrid((tiles_head + tpc - 1) / tpc, heads, 1);
-        for (int r0 = 0; r0 < view.M; r0 += 256) {
-            launch_pdl(tc::score_kernel, sgrid, dim3(tc::kScoreThreads), tc::kScoreSmemBytes, st, map_q_rows, map_k_score, view, plan, r0, std::min(256, view.M - r0),
-                       tpc, scale_log2, (const float *)ws, scores, (int)(r0 > 0), dev_status);
-            if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
-        }
+        if (launch_score_pass(view, plan, map_q_rows, map_k_score, (tiles_head + tpc - 1) / tpc, tpc, scale_log2, ws, scores, dev_status, st, tc::ScoreTileList()) != MAGE_OK)
+            return MAGE_ERR_CUDA;
     }
     if (ev) cudaEventRecord(ev[3], st);
     return MAGE_OK;
@@ -425,6 +437,106 @@ mage_status mage_exact_select_static(const mage_kv_t *kv, const void *q, const v
     }
     return mage_exact_select_events(kv, q, k_blk, v_blk, sm_scale, out, scores, scratch, (size_t)MAGE_STATIC_SCRATCH_BYTES,
                                     dev_status, stream, nullptr);
+}
+
+namespace {
+struct PrunePlan {            // byte offsets into the workspace, after the exact pass's own part
+    int tiles, seeds;         // key tiles per head (by N_max), seed tiles per head
+    size_t rowsum, mass, seed_list, counts, compact, tau, list, list_count, total;
+};
+PrunePlan make_prune_plan(const mage_kv_t *kv, int k) {
+    const Plan plan = make_plan(kv);
+    const size_t heads = (size_t)kv->P * kv->H_kv;
+    PrunePlan pp;
+    pp.tiles = (kv->N_max + 127) / 128;
+    // seed tiles: the heaviest eighth of a head's tiles, and at least twice the k keys the threshold needs.  They are scored in
+    // any case; the threshold they give prunes the rest only if they hold at least k keys that stand out (otherwise it sits
+    // at the background level, every tile passes it and the pass is the dense one)
+    pp.seeds = std::min(pp.tiles, std::max(2 * ((k + 127) / 128), pp.tiles / 8));
+    size_t off = plan.exact_bytes;
+    auto take = [&](size_t bytes) { const size_t at = off; off += align_up(bytes, 256); return at; };
+    pp.rowsum = take(heads * pp.tiles * plan.Mw * sizeof(float2));
+    pp.mass = take(heads * pp.tiles * sizeof(float));
+    pp.seed_list = take(heads * pp.seeds * sizeof(int));
+    pp.counts = take((size_t)kv->P * 3 * sizeof(int));              // seed tiles taken, key tiles, entries of the compact rows: per problem
+    pp.compact = take(heads * pp.seeds * 128 * sizeof(float));
+    pp.tau = take(heads * sizeof(float));
+    pp.list = take(heads * pp.tiles * sizeof(int));
+    pp.list_count = take(heads * sizeof(int));
+    pp.total = off;
+    return pp;
+}
+}  // namespace
+
+size_t mage_pruned_workspace_bytes(const mage_kv_t *kv, int32_t k) {
+    if (!valid_kv(kv, nullptr) || k < 1) return 0;
+    return make_prune_plan(kv, k).total;
+}
+
+mage_status mage_exact_select_pruned(const mage_kv_t *kv, const void *q, const void *k_blk, const void *v_blk, float sm_scale,
+                                     int32_t k, float dense_above, void *out, float *scores, int32_t *indices, int32_t *k_eff,
+                                     int32_t *tiles_scored, void *workspace, size_t workspace_bytes, uint32_t *dev_status,
+                                     void *stream) {
+    mage_status why = MAGE_OK;
+    if (!valid_kv(kv, &why)) return why;
+    if (!q || !k_blk || !v_blk || !out || !indices || !k_eff || !workspace || k < 1 || (kv->N_max > 0 && !scores)) return MAGE_ERR_INVALID_ARG;
+    if (!(sm_scale > 0.f) || !(dense_above >= 0.f) || (reinterpret_cast<uintptr_t>(workspace) & 255)) return MAGE_ERR_INVALID_ARG;
+    if (kv->flags & MAGE_FLAG_SIMT_KERNELS) return MAGE_ERR_UNSUPPORTED;
+    const Plan plan = make_plan(kv);
+    const PrunePlan pp = make_prune_plan(kv, k);
+    if (workspace_bytes < pp.total) return MAGE_ERR_WORKSPACE;
+    const KvView view = make_view(kv);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int heads = kv->P * kv->H_kv;
+    char *wsb = static_cast<char *>(workspace);
+    float *ws = static_cast<float *>(workspace);
+    const __nv_bfloat16 *qb = static_cast<const __nv_bfloat16 *>(q);
+    if (kv->N_max == 0) {                                     // no prefix: attention inside the block, nothing to select
+        const mage_status s = launch_exact_select(kv, view, plan, qb, static_cast<const __nv_bfloat16 *>(k_blk), static_cast<const __nv_bfloat16 *>(v_blk),
+                                                  sm_scale, static_cast<__nv_bfloat16 *>(out), nullptr, ws, dev_status, st, nullptr);
+        if (s != MAGE_OK) return s;
+        if (tiles_scored && cudaMemsetAsync(tiles_scored, 0, (size_t)heads * sizeof(int), st) != cudaSuccess) return MAGE_ERR_CUDA;
+        topk_kernel<<<heads, kTopkThreads, 0, st>>>(scores, kv->seq_lens, kv->H_kv, 0, k, indices, k_eff);
+        return launch_check();
+    }
+    // the score pass's tensor maps first: nothing is launched if they cannot be encoded
+    CUtensorMap map_q_rows, map_k;
+    const mage_status sup = tc_supported(kv);
+    if (sup != MAGE_OK) return sup;
+    if (!tc::make_rows_map(&map_q_rows, q, (long long)kv->P * kv->H_q * kv->B) || !tc::make_cache_map(&map_k, kv, kv->k_cache)) return MAGE_ERR_UNSUPPORTED;
+    float2 *rowsum = reinterpret_cast<float2 *>(wsb + pp.rowsum);
+    float *mass = reinterpret_cast<float *>(wsb + pp.mass), *compact = reinterpret_cast<float *>(wsb + pp.compact), *tau = reinterpret_cast<float *>(wsb + pp.tau);
+    int *seed_list = reinterpret_cast<int *>(wsb + pp.seed_list), *seed_count = reinterpret_cast<int *>(wsb + pp.counts), *tile_counts = seed_count + kv->P,
+        *compact_lens = seed_count + 2 * kv->P, *list = reinterpret_cast<int *>(wsb + pp.list), *list_count = reinterpret_cast<int *>(wsb + pp.list_count);
+    // 1. exact attention; the pass also leaves each tile's row sums behind
+    mage_status s = launch_exact_select(kv, view, plan, qb, static_cast<const __nv_bfloat16 *>(k_blk), static_cast<const __nv_bfloat16 *>(v_blk), sm_scale,
+                                        static_cast<__nv_bfloat16 *>(out), nullptr, ws, dev_status, st, nullptr, false, rowsum, pp.tiles);
+    if (s != MAGE_OK) return s;
+    // 2. tile masses, 3. the seed tiles = the largest masses
+    const long long warps = (long long)heads * pp.tiles;
+    prune::tile_mass_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(view, plan, rowsum, pp.tiles, ws, mass, tile_counts);
+    if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    topk_kernel<<<heads, kTopkThreads, 0, st>>>(mass, tile_counts, kv->H_kv, pp.tiles, pp.seeds, seed_list, seed_count);
+    if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    // 4. exact scores of the seed tiles (also in list order, for the threshold)
+    const float scale_log2 = sm_scale * kLog2e;
+    const int tpc_dense = tc::tiles_per_cta_for(heads, kv->N_max, kv->page_size != 0), tpc = std::max(1, std::min(32, tpc_dense));
+    tc::ScoreTileList seeds;
+    seeds.tiles = seed_list; seeds.count = seed_count; seeds.stride = pp.seeds; seeds.count_per_problem = 1;
+    seeds.compact = compact; seeds.compact_lens = compact_lens;
+    if (launch_score_pass(view, plan, map_q_rows, map_k, (pp.seeds + tpc - 1) / tpc, tpc, scale_log2, ws, scores, dev_status, st, seeds) != MAGE_OK) return MAGE_ERR_CUDA;
+    // 5. tau = the k-th largest seed score (0 if the seeds hold no more than k keys: then nothing is pruned)
+    topk_kernel<<<heads, kTopkThreads, 0, st>>>(compact, compact_lens, kv->H_kv, pp.seeds * 128, k, indices, k_eff, tau);
+    if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    // 6. the further tiles to score; zeros where nothing can be selected
+    prune::mark_kernel<<<heads, 256, (size_t)pp.tiles, st>>>(view, pp.tiles, mass, seed_list, pp.seeds, seed_count, tau, dense_above, list, list_count, scores, tiles_scored);
+    if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    // 7. their exact scores, 8. Top-k of the array
+    tc::ScoreTileList rest;
+    rest.tiles = list; rest.count = list_count; rest.stride = pp.tiles;
+    if (launch_score_pass(view, plan, map_q_rows, map_k, (pp.tiles + tpc - 1) / tpc, tpc, scale_log2, ws, scores, dev_status, st, rest) != MAGE_OK) return MAGE_ERR_CUDA;
+    topk_kernel<<<heads, kTopkThreads, 0, st>>>(scores, kv->seq_lens, kv->H_kv, kv->N_max, k, indices, k_eff);
+    return launch_check();
 }
 
 size_t mage_quest_workspace_bytes(const mage_kv_t *kv, int32_t k) {

@@ -73,6 +73,17 @@ __device__ __forceinline__ bool cache_box_coords(const KvView &kv, int p, int h,
 // warpgroup of a tile hands its 128 partial sums to the row-half-0 warpgroup through shared memory, which adds them
 // (fixed order) one unit late and stores the score.
 // ------------------------------------------------------------------------------------------------------------
+// Optional tile list of the score pass (pruned selection): per (problem, KV head) an ascending list of key-tile numbers to
+// score instead of all tiles.  count is per KV head, or per problem when count_per_problem is set; compact, when given,
+// receives the listed tiles' scores in list order ([P*H_kv][stride][128]) and compact_lens[p] their number of entries.
+struct ScoreTileList {
+    const int *tiles = nullptr;
+    const int *count = nullptr;
+    int stride = 0, count_per_problem = 0;
+    float *compact = nullptr;
+    int *compact_lens = nullptr;
+};
+
 constexpr int kScoreStages = 4;
 constexpr int kScoreWgs = 4;
 constexpr int kScoreThreads = kScoreWgs * 128 + 64;
@@ -83,16 +94,20 @@ constexpr size_t kScoreSmemBytes = 1024 + kScoreQBytes + kScoreStages * kTileByt
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, KvView kv, Plan plan,
              int row_begin, int rows, int tiles_per_cta, float scale_log2, const float *__restrict__ ws,
-             float *__restrict__ scores, int accumulate, unsigned *status) {
+             float *__restrict__ scores, int accumulate, unsigned *status, ScoreTileList list) {
     using namespace ptx;
     pdl_wait();
     pdl_launch_dependents();
     const int z = blockIdx.y, p = z / kv.H_kv, h = z % kv.H_kv;
     const int N = seq_len_of(kv, p);
-    const int tiles_total = (N + kTile - 1) / kTile;
+    // list mode (pruned selection): the CTA walks entries [tile0, tile0 + n_my) of this head's ascending list of tile numbers
+    const int *my_list = list.tiles ? list.tiles + (size_t)z * list.stride : nullptr;
+    const int tiles_total = my_list ? min(list.count[list.count_per_problem ? p : z], list.stride) : (N + kTile - 1) / kTile;
     const int tile0 = blockIdx.x * tiles_per_cta;
+    if (my_list && blockIdx.x == 0 && h == 0 && threadIdx.x == 0 && list.compact_lens) list.compact_lens[p] = tiles_total * kTile;
     if (tile0 >= tiles_total) return;
     const int n_my = min(tiles_per_cta, tiles_total - tile0);
+    auto tile_of = [&](int t) { return my_list ? my_list[tile0 + t] : tile0 + t; };     // actual key tile of the CTA's t-th
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -146,7 +161,7 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
             for (int i = 0; i < n_my; ++i) {
                 const int slot = i % kScoreStages, u = i / kScoreStages;
                 if (!mbar_wait(bar(EMPTY + slot), (u & 1) ^ 1, abort_s, status)) break;
-                const int j0 = (tile0 + i) * kTile;
+                const int j0 = tile_of(i) * kTile;
                 int c1[2], c2[2], c3[2], bad = 0;
                 for (int kh = 0; kh < 2; ++kh)
                     if (cache_box_coords(kv, p, h, j0 + kh * 64, N, c1[kh], c2[kh], c3[kh], status)) bad |= 1 << kh;
@@ -210,8 +225,12 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                 mbar_arrive_warp(bar(P_EMPTY + par));
             }
             v = bad ? 0.f : v * inv_m;
-            const int j = (tile0 + t) * kTile + key;
+            const int j = tile_of(t) * kTile + key;
             if (j < N) srow[j] = accumulate ? srow[j] + v : v;
+            if (list.compact) {                                  // the same scores in list order, zeros past the prefix
+                float *c = list.compact + ((size_t)z * list.stride + tile0 + t) * kTile + key;
+                *c = j < N ? (accumulate ? *c + v : v) : 0.f;
+            }
             return true;
         };
         bool ok = true;
@@ -382,6 +401,11 @@ __device__ __noinline__ uint32_t sparse_bad_cols(const int *row_tab, const int *
 struct AttnMaps {
     CUtensorMap q, k, v, kb, vb;
     int gather_rows = 0, gather_blk_rows = 0, gather_pitch = 0, lse_only = 0;
+    // exact pass only, optional: per (KV head, 128-key tile, query row) the tile's unnormalised row sum and the reference it
+    // was taken against, [P*H_kv][rowsum_tiles][Mw] pairs; sum * 2^(reference - row's log2-sum-exp) is the row's probability
+    // mass on that tile, which the pruned selection adds up over rows into an upper bound for every key of the tile
+    float2 *rowsum = nullptr;
+    int rowsum_tiles = 0;
     int test_stall = 0;          // MAGE_FLAG_TEST_STALL: the exact pass never requests its first key tile and waits with the short limit
 };
 
@@ -857,6 +881,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 };
                 // a warp whose 32 rows all lie beyond M (row padding of the last M-tile) only takes part in the hand-offs
                 bool fast = valid == kTile && bad == 0, half_done = false;
+                float tile_sum = 0.f;                      // this tile's part of l, relative to m_used as it stands after the tile
                 if (warp_has_rows && fast && i == first) {
                     // first tile: the reference starts at the maximum of the row's first 32 logits; the sweep below moves it
                     // on lazily like any later rise (and redoes the tile on the careful path if the rest of the row lies
@@ -951,6 +976,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                                 for (int e = 0; e < 16; ++e) l_first += __uint_as_float(pr[e] << 16) + __uint_as_float(pr[e] & 0xffff0000u);
                             }
                             l += l_first * f;
+                            tile_sum = l_first * f;
                             m_used = m_new;
                             neg_m2 = pack2(-m_used, -m_used);
                             l2a = pack2(0.f, 0.f);
@@ -970,6 +996,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                         unpack2(l2a, a0, a1);
                         unpack2(l2b, b0, b1);
                         l += (a0 + a1) + (b0 + b1);
+                        tile_sum += (a0 + a1) + (b0 + b1);
                         if (mx > kRescaleThreshold) { pending = true; pend_m = m_used + mx; }
                         tmem_st16(tS + 32, pa);
                         tmem_st16(tS + 48, pb);
@@ -1046,7 +1073,10 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                         tmem_st16(tS + (c0 >> 1), pk);
                     }
                     l += l0 + l1;
+                    tile_sum = l0 + l1;
                 }
+                if (!SPARSE && maps.rowsum != nullptr && !blk_chunk && grow < kv.M)
+                    maps.rowsum[((size_t)z * maps.rowsum_tiles + (j_begin / kTile + i)) * plan.Mw + grow] = make_float2(tile_sum, m_used);
                 tmem_wait_st();
                 if (!SPARSE && valid != kTile && (tp || mt == 0)) {
                     // Last tile of the prefix: cache rows past the end may hold anything (even NaN patterns), and

@@ -17,9 +17,11 @@ __device__ __forceinline__ unsigned float_order_key(float f) {
 //     and how many entries equal to T are still needed;
 //  2. one ordered pass emits every position with key > T and the first `need_eq` positions with key == T,
 //     placed by a block-wide prefix sum, so the output is ascending and ties go to the smaller position.
+// kth_out (optional, [P*H_kv]): the k_eff-th largest score of the row, or 0 when the row has no more than k entries.
 __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *__restrict__ scores,
                                                             const int *__restrict__ seq_lens, int H_kv, int N_max,
-                                                            int k, int *__restrict__ indices, int *__restrict__ k_eff_out) {
+                                                            int k, int *__restrict__ indices, int *__restrict__ k_eff_out,
+                                                            float *__restrict__ kth_out = nullptr) {
     __shared__ unsigned hist4[4][2048];
     __shared__ unsigned hist[32];
     __shared__ unsigned warp_tot[32];
@@ -32,6 +34,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *__restr
     const float *s = scores + (size_t)z * N_max;
     int *out = indices + (size_t)z * k;
     if (h == 0 && tid == 0) k_eff_out[p] = k_eff;
+    if (kth_out && tid == 0) kth_out[z] = 0.f;           // rows with no more than k entries have no threshold
     for (int t = k_eff + tid; t < k; t += kTopkThreads) out[t] = -1;
     if (k_eff == 0) return;
     if (k_eff == N) {
@@ -104,6 +107,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *__restr
         __syncthreads();
     }
     const unsigned T = prefix, need_eq = need;
+    if (kth_out && tid == 0) kth_out[z] = __uint_as_float((T & 0x80000000u) ? (T & 0x7fffffffu) : ~T);
 
     // Ordered emit.  A stretch of 32 x span entries at a time (span = 4096, less for short rows so that every warp has a
     // share): warp w owns entries [w * span, (w + 1) * span) of the stretch, lane l the four entries at 128 * i + 4 * l of
