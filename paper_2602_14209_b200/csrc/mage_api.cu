@@ -369,6 +369,26 @@ mage_status mage_topk(const float *scores, const int32_t *seq_lens, int32_t P, i
                       int32_t *indices, int32_t *k_eff, void *workspace, size_t workspace_bytes, void *stream) {
     (void)workspace; (void)workspace_bytes;
     if (P < 1 || H_kv < 1 || N_max < 0 || k < 1 || !indices || !k_eff || (N_max > 0 && !scores)) return MAGE_ERR_INVALID_ARG;
+    // long rows of a few heads: a cluster of eight CTAs per head shares the row; otherwise one CTA per head
+    // (few heads only: a cluster member costs a whole SM for about 25 us whatever the row length, so with many heads the
+    // single-CTA kernel, one SM per head, finishes sooner)
+    if (N_max >= 16384 && P * H_kv * kTopkCluster <= 148) {
+        if (opt_in_smem(topk_cluster_kernel, kTopkClusterSmem) != MAGE_OK) return MAGE_ERR_CUDA;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(kTopkCluster, P * H_kv, 1);
+        cfg.blockDim = dim3(kTopkThreads);
+        cfg.dynamicSmemBytes = kTopkClusterSmem;
+        cfg.stream = static_cast<cudaStream_t>(stream);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = kTopkCluster;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaLaunchKernelEx(&cfg, topk_cluster_kernel, scores, seq_lens, H_kv, N_max, k, indices, k_eff);
+        return launch_check();
+    }
     topk_kernel<<<P * H_kv, kTopkThreads, 0, static_cast<cudaStream_t>(stream)>>>(scores, seq_lens, H_kv, N_max, k, indices, k_eff);
     return launch_check();
 }
@@ -598,6 +618,7 @@ const char *mage_status_string(mage_status s) {
 uint64_t mage_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 #ifdef MAGE_TIMING
+int mage_debug_topk_stamps(unsigned long long *host_out) { return (int)cudaMemcpyFromSymbol(host_out, g_topk_stamps, sizeof(unsigned long long) * 64); }
 int mage_debug_stamps(unsigned long long *host_out) { return (int)cudaMemcpyFromSymbol(host_out, tc::g_stamps, sizeof(unsigned long long) * 128); }
 #endif
 

@@ -197,4 +197,261 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *__restr
     }
 }
 
+
+// ------------------------------------------------------------------------------------------------------------
+// The same selection with a cluster of eight CTAs per (problem, KV head), for long rows: CTA c owns the c-th eighth of
+// the row and keeps it in shared memory, so the scores are read from L2 once instead of once per pass, by eight SMs
+// instead of one.  The CTAs meet through distributed shared memory (plain remote loads and stores): per radix pass every
+// CTA publishes its digit histogram in its own shared memory, one cluster barrier, and every CTA adds up the eight
+// histograms and takes the same decision; before the ordered emit the CTAs exchange how many selected entries each holds.  Exact and deterministic like the single-CTA kernel, same output.
+// ------------------------------------------------------------------------------------------------------------
+constexpr int kTopkCluster = 8;
+constexpr int kTopkSliceCap = 40960;                    // floats of a CTA's share kept in shared memory (160 KB)
+constexpr size_t kTopkClusterSmem = 7 * 2048 * sizeof(unsigned) + (size_t)kTopkSliceCap * sizeof(float);
+
+#ifdef MAGE_TIMING
+__device__ unsigned long long g_topk_stamps[64];
+#define TOPK_STAMP(i) do { if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_topk_stamps[i] = t_; } } while (0)
+#else
+#define TOPK_STAMP(i) ((void)0)
+#endif
+
+namespace cl {
+__device__ __forceinline__ unsigned cta_rank() { unsigned r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ unsigned map_to(const void *smem_ptr, unsigned rank) {         // this CTA's address -> CTA `rank`'s
+    unsigned a = static_cast<unsigned>(__cvta_generic_to_shared(smem_ptr)), r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ unsigned ld_u32(unsigned addr) { unsigned v; asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory"); return v; }
+// every thread of every CTA of the cluster; orders the remote accesses before it against those after it
+__device__ __forceinline__ void sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+}  // namespace cl
+
+__global__ void __launch_bounds__(kTopkThreads) topk_cluster_kernel(const float *__restrict__ scores, const int *__restrict__ seq_lens,
+                                                                    int H_kv, int N_max, int k, int *__restrict__ indices,
+                                                                    int *__restrict__ k_eff_out) {
+    extern __shared__ __align__(16) unsigned char dyn_s[];
+    unsigned (*hist4)[2048] = reinterpret_cast<unsigned (*)[2048]>(dyn_s);                                // [4][2048]
+    unsigned (*mine)[2048] = reinterpret_cast<unsigned (*)[2048]>(dyn_s + 4 * 2048 * sizeof(unsigned));   // [3][2048]: this CTA's digit counts of each pass, read by its peers
+    float *slice_s = reinterpret_cast<float *>(dyn_s + 7 * 2048 * sizeof(unsigned));
+    __shared__ unsigned merged[3][256];                  // digits [256 c, 256 c + 256) summed over the cluster, per pass
+    __shared__ unsigned counts[2];                       // selected (greater, equal) entries this CTA holds, read by the CTAs after it
+    __shared__ unsigned hist[32], warp_tot[32];
+    __shared__ unsigned sel_digit, sel_need;
+
+    TOPK_STAMP(0);
+    const unsigned c = cl::cta_rank();
+    const int z = blockIdx.y, p = z / H_kv, h = z % H_kv, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int N = seq_lens ? seq_lens[p] : N_max;
+    N = N < 0 ? 0 : (N > N_max ? N_max : N);
+    const int k_eff = k < N ? k : N;
+    const float *row = scores + (size_t)z * N_max;
+    int *out = indices + (size_t)z * k;
+    // the trivial cases are the same for every CTA of the cluster: all of them leave before the first cluster barrier
+    if (k_eff == 0 || k_eff == N) {
+        if (c == 0) {
+            if (h == 0 && tid == 0) k_eff_out[p] = k_eff;
+            for (int t = tid; t < k; t += kTopkThreads) out[t] = t < k_eff ? t : -1;
+        }
+        return;
+    }
+    if (c == 0) {
+        if (h == 0 && tid == 0) k_eff_out[p] = k_eff;
+        for (int t = k_eff + tid; t < k; t += kTopkThreads) out[t] = -1;
+    }
+    // this CTA's share [lo, lo + n) of the row, a multiple of four entries long
+    const int share = (((N + kTopkCluster - 1) / kTopkCluster) + 3) & ~3;
+    const int lo = min(N, (int)c * share), n = min(N, lo + share) - lo;
+    const bool vec_ok = (reinterpret_cast<uintptr_t>(row) & 15) == 0;
+    const bool cached = share <= kTopkSliceCap;
+    if (cached) {
+        for (int j = tid * 4; j < n; j += kTopkThreads * 4) {
+            if (vec_ok && j + 3 < n) {
+                *reinterpret_cast<float4 *>(slice_s + j) = *reinterpret_cast<const float4 *>(row + lo + j);
+            } else {
+                for (int e = 0; e < 4 && j + e < n; ++e) slice_s[j + e] = row[lo + j + e];
+            }
+        }
+    }
+    TOPK_STAMP(1);
+    const float *s = cached ? slice_s : row + lo;
+    const bool s_vec = cached || vec_ok;
+    __syncthreads();
+    TOPK_STAMP(2);
+
+    auto for_each = [&](auto &&body) {
+        for (int base = 0; base < n; base += kTopkThreads * 16) {
+            float v[16];
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+                const int j = base + q4 * kTopkThreads * 4 + tid * 4;
+                if (s_vec && j + 3 < n) {
+                    const float4 f = *reinterpret_cast<const float4 *>(s + j);
+                    v[q4 * 4 + 0] = f.x; v[q4 * 4 + 1] = f.y; v[q4 * 4 + 2] = f.z; v[q4 * 4 + 3] = f.w;
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) v[q4 * 4 + e] = j + e < n ? s[j + e] : 0.f;
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                const int j = base + (e >> 2) * kTopkThreads * 4 + tid * 4 + (e & 3);
+                if (j < n) body(float_order_key(v[e]));
+            }
+        }
+    };
+
+    unsigned prefix = 0u, mask = 0u, need = (unsigned)k_eff;
+#pragma unroll 1
+    for (int pass = 0; pass < 3; ++pass) {
+        const int lob = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+        const unsigned dmask = pass == 2 ? 1023u : 2047u;
+        for (int t = tid; t < 4 * 2048; t += kTopkThreads) (&hist4[0][0])[t] = 0;
+        __syncthreads();
+        unsigned *my_hist = hist4[warp & 3];
+        for_each([&](unsigned key) {
+            if ((key & mask) == prefix) atomicAdd(&my_hist[(key >> lob) & dmask], 1u);
+        });
+        __syncthreads();
+        TOPK_STAMP(3 + 4 * pass);
+        // this CTA's counts of the digits 2 * tid, 2 * tid + 1 are published in its own shared memory; after the barrier every
+        // CTA reads all eight CTAs' counts of its threads' digits (sixteen remote loads in flight at once) and adds them up
+        mine[pass][2 * tid] = hist4[0][2 * tid] + hist4[1][2 * tid] + hist4[2][2 * tid] + hist4[3][2 * tid];
+        mine[pass][2 * tid + 1] = hist4[0][2 * tid + 1] + hist4[1][2 * tid + 1] + hist4[2][2 * tid + 1] + hist4[3][2 * tid + 1];
+        TOPK_STAMP(4 + 4 * pass);
+        cl::sync_all();
+        TOPK_STAMP(5 + 4 * pass);
+        // two steps, so that a CTA makes 4096 remote loads per pass instead of 16384: CTA c adds up digits [256 c, 256 c + 256)
+        // over the eight CTAs and publishes the sums; after a second barrier every thread fetches its two digits' sums
+        if (tid < 256) {
+            unsigned part[kTopkCluster];
+#pragma unroll
+            for (int cc = 0; cc < kTopkCluster; ++cc) part[cc] = cl::ld_u32(cl::map_to(&mine[pass][256 * c + tid], cc));
+            unsigned sum = 0;
+#pragma unroll
+            for (int cc = 0; cc < kTopkCluster; ++cc) sum += part[cc];
+            merged[pass][tid] = sum;
+        }
+        cl::sync_all();
+        const unsigned owner = cl::map_to(&merged[pass][(2 * tid) & 255], (unsigned)(2 * tid) >> 8);
+        const unsigned c0 = cl::ld_u32(owner), c1 = cl::ld_u32(owner + 4);
+        unsigned v = c0 + c1;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned dn = __shfl_down_sync(0xffffffffu, v, off);
+            if (lane + off < 32) v += dn;
+        }
+        if (lane == 0) warp_tot[warp] = v;
+        __syncthreads();
+        unsigned above = 0;
+        for (int w = warp + 1; w < 32; ++w) above += warp_tot[w];
+        const unsigned ge0 = v + above, ge1 = ge0 - c0, ge2 = ge1 - c1;
+        if (ge1 >= need && ge2 < need) { sel_digit = 2 * tid + 1; sel_need = need - ge2; }
+        else if (ge0 >= need && ge1 < need) { sel_digit = 2 * tid; sel_need = need - ge1; }
+        __syncthreads();
+        prefix |= sel_digit << lob;
+        mask |= dmask << lob;
+        need = sel_need;
+        __syncthreads();
+        TOPK_STAMP(6 + 4 * pass);
+    }
+    const unsigned T = prefix, need_eq = need;
+
+    // Ordered emit.  Thread t owns 16 consecutive entries of each 16384-entry stretch of the share.  First sweep: how many
+    // entries above / equal to the threshold the CTA holds, published for the CTAs after it; second sweep: a block-wide
+    // prefix sum places each thread's entries.  Ties go to the smaller position: an equal entry is written only while
+    // fewer than need_eq equal entries precede it in the row.
+    auto masks_of = [&](int base, unsigned &gt, unsigned &eq) {
+        gt = eq = 0;
+        const int j0 = base + tid * 16;
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+            float v[4];
+            const int j = j0 + q4 * 4;
+            if (s_vec && j + 3 < n) {
+                const float4 f = *reinterpret_cast<const float4 *>(s + j);
+                v[0] = f.x; v[1] = f.y; v[2] = f.z; v[3] = f.w;
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) v[e] = j + e < n ? s[j + e] : 0.f;
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                if (j + e < n) {
+                    const unsigned key = float_order_key(v[e]);
+                    gt |= (unsigned)(key > T) << (q4 * 4 + e);
+                    eq |= (unsigned)(key == T) << (q4 * 4 + e);
+                }
+            }
+        }
+    };
+    unsigned my_gt = 0, my_eq = 0;
+    for (int base = 0; base < n; base += kTopkThreads * 16) {
+        unsigned gt, eq;
+        masks_of(base, gt, eq);
+        my_gt += __popc(gt);
+        my_eq += __popc(eq);
+    }
+    my_gt = __reduce_add_sync(0xffffffffu, my_gt);
+    my_eq = __reduce_add_sync(0xffffffffu, my_eq);
+    if (lane == 0) { warp_tot[warp] = my_gt; hist[warp] = my_eq; }
+    __syncthreads();
+    if (warp == 0) {
+        const unsigned g = __reduce_add_sync(0xffffffffu, warp_tot[lane]), e = __reduce_add_sync(0xffffffffu, hist[lane]);
+        if (lane == 0) { counts[0] = g; counts[1] = e; }
+    }
+    TOPK_STAMP(20);
+    cl::sync_all();
+    TOPK_STAMP(21);
+    unsigned run_gt = 0, run_eq = 0;                      // selected entries before this CTA's share
+    for (unsigned cc = 0; cc < c; ++cc) {
+        run_gt += cl::ld_u32(cl::map_to(&counts[0], cc));
+        run_eq += cl::ld_u32(cl::map_to(&counts[1], cc));
+    }
+    for (int base = 0; base < n; base += kTopkThreads * 16) {
+        unsigned gt, eq;
+        masks_of(base, gt, eq);
+        const unsigned packed = ((unsigned)__popc(gt) << 16) | (unsigned)__popc(eq);
+        unsigned incl = packed;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned up = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += up;
+        }
+        __syncthreads();                                  // warp_tot is free again
+        if (lane == 31) warp_tot[warp] = incl;
+        __syncthreads();
+        unsigned before = 0, total = 0;
+        for (int w = 0; w < 32; ++w) {
+            const unsigned wt = warp_tot[w];
+            before += w < warp ? wt : 0u;
+            total += wt;
+        }
+        const unsigned excl = before + incl - packed;
+        unsigned g = run_gt + (excl >> 16), q = run_eq + (excl & 0xffffu);
+        if (gt | eq) {
+            const int j0 = lo + base + tid * 16;
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                if (gt & (1u << e)) {
+                    out[g + min(q, need_eq)] = j0 + e;
+                    ++g;
+                } else if (eq & (1u << e)) {
+                    if (q < need_eq) out[g + q] = j0 + e;
+                    ++q;
+                }
+            }
+        }
+        run_gt += total >> 16;
+        run_eq += total & 0xffffu;
+    }
+    TOPK_STAMP(22);
+    cl::sync_all();                                       // CTA 0's shared memory stays until every CTA has read it
+    TOPK_STAMP(23);
+}
+
 }  // namespace mage
