@@ -59,6 +59,23 @@ __device__ __forceinline__ bool cache_box_coords(const KvView &kv, int p, int h,
     return false;
 }
 
+// Paged caches: the page-table entry of the 64-key box at logical position j (-2 beyond the prefix), and the box
+// coordinates from an entry looked up earlier.  The producers look entries up a tile or two ahead of their use: a lookup
+// is a dependent global load of about half a microsecond, and four of them per tile (two boxes each of K and V) on the
+// producer's critical path would take longer than the tile's arithmetic.
+__device__ __forceinline__ int page_entry(const KvView &kv, int p, int j, int N) {
+    return j < N ? kv.block_table[(long long)p * kv.max_pages + j / kv.page_size] : -2;
+}
+__device__ __forceinline__ bool paged_box_coords(const KvView &kv, int h, int j, int entry, int &c1, int &c2, int &c3, unsigned *status) {
+    c1 = j % kv.page_size;
+    c2 = h;
+    c3 = kv.num_pages;                     // out of range: zero fill
+    if (entry == -2) return false;         // beyond the prefix
+    if (entry >= 0 && entry < kv.num_pages) { c3 = entry; return false; }
+    if (status) atomicOr(status, MAGE_DEV_BAD_PAGE);
+    return true;
+}
+
 // ------------------------------------------------------------------------------------------------------------
 // Block-score kernel (Eq. 4): score[j] = 1/M * sum_r exp2(scale_log2 * <q_r, k_j> - lse2_r).
 // Orientation: keys are the MMA M dimension (TMEM lanes), query rows the N dimension (TMEM columns), so each
@@ -157,15 +174,31 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                 for (int rb = 0; rb < rows64 / 64; ++rb)
                     tma_load_2d(smem_u32(q_s + dh * (kScoreQBytes / 2) + rb * kBoxBytes), &map_q, bar(Q_FULL), dh * 64, q_row0 + rb * 64);
             const uint64_t pol_k = l2_policy_evict_first();       // last use of these K lines
+            const bool paged = kv.page_size != 0;
+            int pg_cur[2] = {-2, -2}, pg_nxt[2] = {-2, -2};        // page-table entries of the CTA's tile i and tile i + 1
+            if (paged) {
+                for (int kh = 0; kh < 2; ++kh) {
+                    pg_cur[kh] = page_entry(kv, p, tile_of(0) * kTile + kh * 64, N);
+                    pg_nxt[kh] = n_my > 1 ? page_entry(kv, p, tile_of(1) * kTile + kh * 64, N) : -2;
+                }
+            }
             int issued = 0;
             for (int i = 0; i < n_my; ++i) {
                 const int slot = i % kScoreStages, u = i / kScoreStages;
                 if (!mbar_wait(bar(EMPTY + slot), (u & 1) ^ 1, abort_s, status)) break;
                 const int j0 = tile_of(i) * kTile;
                 int c1[2], c2[2], c3[2], bad = 0;
-                for (int kh = 0; kh < 2; ++kh)
-                    if (cache_box_coords(kv, p, h, j0 + kh * 64, N, c1[kh], c2[kh], c3[kh], status)) bad |= 1 << kh;
-                if (kv.page_size != 0) tile_bad_s[i & 15] = bad;       // ordered before the tile's FULL phase by the arrive below
+                if (paged) {
+                    for (int kh = 0; kh < 2; ++kh)
+                        if (paged_box_coords(kv, h, j0 + kh * 64, pg_cur[kh], c1[kh], c2[kh], c3[kh], status)) bad |= 1 << kh;
+                    tile_bad_s[i & 15] = bad;                         // ordered before the tile's FULL phase by the arrive below
+                    for (int kh = 0; kh < 2; ++kh) {
+                        pg_cur[kh] = pg_nxt[kh];
+                        pg_nxt[kh] = i + 2 < n_my ? page_entry(kv, p, tile_of(i + 2) * kTile + kh * 64, N) : -2;
+                    }
+                } else {
+                    for (int kh = 0; kh < 2; ++kh) cache_box_coords(kv, p, h, j0 + kh * 64, N, c1[kh], c2[kh], c3[kh], nullptr);
+                }
                 mbar_arrive_expect_tx(bar(FULL + slot), kTileBytes);
                 for (int kh = 0; kh < 2; ++kh)
                     for (int dh = 0; dh < 2; ++dh)
@@ -546,34 +579,64 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 // of a 32K prefix: 32 MB, it does; a 28-layer 128K batch streams 3.8 GB of K, it does not).
                 const uint64_t pol_k = l2_policy_evict_last(), pol_v = l2_policy_evict_first();
                 int issued = 0;
-                for (int L = 0; L < 2 * n_tiles; ++L) {
-                    const int i = L >> 1, is_v = L & 1, slot = slot_of(L);
-                    if (!mbar_wait(bar(EMPTY + slot), par_of(L) ^ 1, abort_s, status)) break;
-                    if (maps.test_stall) break;                // test hook: K(0) is never requested, so nothing is in flight
-                    if (maps.lse_only && is_v) {               // no values in this mode: the slot's phase is completed empty-handed
-                        mbar_arrive(bar(FULL + slot));
-                        issued = L + 1;
-                        continue;
-                    }
-                    int c1[2], c2[2], c3[2], bad = 0;
-                    if (!blk_chunk) {
-                        for (int kh = 0; kh < 2; ++kh)
-                            if (cache_box_coords(kv, p, h, j_begin + i * kTile + kh * 64, N, c1[kh], c2[kh], c3[kh], is_v ? nullptr : status)) bad |= 1 << kh;
-                        if (kv.page_size != 0 && !is_v) tile_bad_s[i & 7] = bad;    // ordered before K(i)'s FULL phase by the arrive below
-                    }
-                    mbar_arrive_expect_tx(bar(FULL + slot), kTileBytes);
-                    const uint32_t dst = smem_u32(kv_s + slot * kTileBytes);
+                if (kv.page_size != 0 && !blk_chunk) {
+                    // paged cache: page-table entries of tile i and tile i + 1 are held in registers, looked up a tile ahead
+                    int pg_cur[2], pg_nxt[2];
                     for (int kh = 0; kh < 2; ++kh) {
-                        if (!blk_chunk) {
-                            for (int dh = 0; dh < 2; ++dh)
-                                tma_load_4d_hint(dst + dh * kHalfBytes + kh * kBoxBytes, is_v ? &maps.v : &maps.k, bar(FULL + slot), dh * 64, c1[kh], c2[kh], c3[kh], is_v ? pol_v : pol_k);
-                        } else {
-                            const int row = (i == 0 && kh == 0) ? z * kv.B : blk_rows_total + 64;   // beyond the tensor: zero fill
-                            for (int dh = 0; dh < 2; ++dh)
-                                tma_load_2d(dst + dh * kHalfBytes + kh * kBoxBytes, is_v ? &maps.vb : &maps.kb, bar(FULL + slot), dh * 64, row);
-                        }
+                        pg_cur[kh] = page_entry(kv, p, j_begin + kh * 64, N);
+                        pg_nxt[kh] = page_entry(kv, p, j_begin + kTile + kh * 64, N);
                     }
-                    issued = L + 1;
+                    for (int L = 0; L < 2 * n_tiles; ++L) {
+                        const int i = L >> 1, is_v = L & 1, slot = slot_of(L);
+                        if (!mbar_wait(bar(EMPTY + slot), par_of(L) ^ 1, abort_s, status)) break;
+                        if (maps.test_stall) break;            // test hook: K(0) is never requested, so nothing is in flight
+                        if (maps.lse_only && is_v) {           // no values in this mode: the slot's phase is completed empty-handed
+                            mbar_arrive(bar(FULL + slot));
+                        } else {
+                            int c1[2], c2[2], c3[2], bad = 0;
+                            for (int kh = 0; kh < 2; ++kh)
+                                if (paged_box_coords(kv, h, j_begin + i * kTile + kh * 64, pg_cur[kh], c1[kh], c2[kh], c3[kh], is_v ? nullptr : status)) bad |= 1 << kh;
+                            if (!is_v) tile_bad_s[i & 7] = bad;     // ordered before K(i)'s FULL phase by the arrive below
+                            mbar_arrive_expect_tx(bar(FULL + slot), kTileBytes);
+                            const uint32_t dst = smem_u32(kv_s + slot * kTileBytes);
+                            for (int kh = 0; kh < 2; ++kh)
+                                for (int dh = 0; dh < 2; ++dh)
+                                    tma_load_4d_hint(dst + dh * kHalfBytes + kh * kBoxBytes, is_v ? &maps.v : &maps.k, bar(FULL + slot), dh * 64, c1[kh], c2[kh], c3[kh], is_v ? pol_v : pol_k);
+                        }
+                        if (is_v) {                            // tile i + 1 becomes current, tile i + 2 is looked up
+                            for (int kh = 0; kh < 2; ++kh) {
+                                pg_cur[kh] = pg_nxt[kh];
+                                pg_nxt[kh] = page_entry(kv, p, j_begin + (i + 2) * kTile + kh * 64, N);
+                            }
+                        }
+                        issued = L + 1;
+                    }
+                } else {
+                    for (int L = 0; L < 2 * n_tiles; ++L) {
+                        const int i = L >> 1, is_v = L & 1, slot = slot_of(L);
+                        if (!mbar_wait(bar(EMPTY + slot), par_of(L) ^ 1, abort_s, status)) break;
+                        if (maps.test_stall) break;            // test hook: K(0) is never requested, so nothing is in flight
+                        if (maps.lse_only && is_v) {           // no values in this mode: the slot's phase is completed empty-handed
+                            mbar_arrive(bar(FULL + slot));
+                            issued = L + 1;
+                            continue;
+                        }
+                        mbar_arrive_expect_tx(bar(FULL + slot), kTileBytes);
+                        const uint32_t dst = smem_u32(kv_s + slot * kTileBytes);
+                        for (int kh = 0; kh < 2; ++kh) {
+                            if (!blk_chunk) {
+                                int c1, c2, c3;
+                                cache_box_coords(kv, p, h, j_begin + i * kTile + kh * 64, N, c1, c2, c3, nullptr);
+                                for (int dh = 0; dh < 2; ++dh)
+                                    tma_load_4d_hint(dst + dh * kHalfBytes + kh * kBoxBytes, is_v ? &maps.v : &maps.k, bar(FULL + slot), dh * 64, c1, c2, c3, is_v ? pol_v : pol_k);
+                            } else {
+                                const int row = (i == 0 && kh == 0) ? z * kv.B : blk_rows_total + 64;   // beyond the tensor: zero fill
+                                for (int dh = 0; dh < 2; ++dh)
+                                    tma_load_2d(dst + dh * kHalfBytes + kh * kBoxBytes, is_v ? &maps.vb : &maps.kb, bar(FULL + slot), dh * 64, row);
+                            }
+                        }
+                        issued = L + 1;
+                    }
                 }
                 if (*abort_s) {
                     for (int L = max(0, issued - kAttnSlots); L < issued; ++L) {
