@@ -144,7 +144,11 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int rows64 = (rows + 63) & ~63;
     // the two row halves: [0, rows_lo) and [rows_lo, rows); rows_lo is a multiple of 8 rows (one swizzle atom)
-    const int rows_lo = min(rows, (((rows + 1) >> 1) + 7) & ~7), rows_hi = rows - rows_lo;
+    // With at most 128 query rows (e.g. G = 4, B = 32) a unit is a whole tile instead: the four warpgroups take the tiles
+    // i = 0, 1, 2, 3 (mod 4), each with all the rows, and nothing is exchanged between warpgroups ("quad" mode).  Half-row
+    // units of 64 columns would spend as long in their hand-offs as in their exponentials.
+    const bool quad = rows <= 128;
+    const int rows_lo = quad ? rows : min(rows, (((rows + 1) >> 1) + 7) & ~7), rows_hi = rows - rows_lo;
     const int n_units = rows_hi > 0 ? 2 : 1;           // units per tile
 
     if (tid < 16) tile_bad_s[tid] = 0;
@@ -222,7 +226,7 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                 if (!mbar_wait(bar(FULL + slot), su & 1, abort_s, status)) break;
                 const uint32_t k_addr = smem_u32(k_s + slot * kTileBytes), q_addr = smem_u32(q_s);
                 for (int rh = 0; rh < n_units && ok; ++rh) {
-                    const int buf = (i & 1) * 2 + rh, use = i >> 1;          // buffer = warpgroup that consumes it
+                    const int buf = quad ? (i & 3) : (i & 1) * 2 + rh, use = quad ? i >> 2 : i >> 1;     // buffer = warpgroup that consumes it
                     if (!mbar_wait(bar(T_EMPTY + buf), (use & 1) ^ 1, abort_s, status)) { ok = false; break; }
                     tc_fence_after_sync();
 #pragma unroll
@@ -239,7 +243,8 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
         }
     } else {
         const int wg = warp >> 2, w4 = warp & 3, key = w4 * 32 + lane;
-        const int par = wg >> 1, rh = wg & 1;               // tile parity and row half of this warpgroup
+        const int par = quad ? wg : wg >> 1, rh = quad ? 0 : wg & 1;      // tiles i = par (mod step) and row half of this warpgroup
+        const int step = quad ? 4 : 2;
         const float inv_m = 1.f / (float)kv.M;
         float *srow = scores + (size_t)z * kv.N_max;
         const int col_lo = rh ? rows_lo : 0, n_cols = rh ? rows_hi : rows_lo;      // my columns: neg_lse index = col_lo + c
@@ -268,8 +273,8 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
         };
         bool ok = true;
         if (n_cols > 0) {
-            for (int i = par; i < n_my; i += 2) {
-                const int use = i >> 1;
+            for (int i = par; i < n_my; i += step) {
+                const int use = quad ? i >> 2 : i >> 1;
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(T_FULL + wg), use & 1, abort_s, status))) { ok = false; break; }
                 tc_fence_after_sync();
                 const bool key_bad = (tile_bad_s[i & 15] >> (key >> 6)) & 1;
