@@ -98,8 +98,9 @@ class BlockAttention:
         o = self.exact_select(q_steps[0], kb_steps[0], vb_steps[0], None if outs is None else outs[0], events=events)
         res.append(o)
         self.select_async()
-        if T > 1:
-            self.join()
+        # joined even when no reuse step follows (T = 1): the index sets and k_eff are then ordered with respect to the main
+        # stream for the caller, and the next block's Step 1 cannot overwrite the scores while top-k still reads them
+        self.join()
         for t in range(1, T):
             res.append(self.sparse_step(q_steps[t], kb_steps[t], vb_steps[t], None if outs is None else outs[t]))
         return res
@@ -154,8 +155,7 @@ class HostStagedBlocks:
             ba.exact_select(self.q_s[b][0], self.kb_s[b][0], self.vb_s[b][0], self.out_s[b][0])
             ba.select_async(main)
             self.ev_out[b][0].record(main)
-            if T > 1:
-                ba.join(main)
+            ba.join(main)
             for t in range(1, T):
                 main.wait_event(self.ev_in[b][t])
                 ba.sparse_step(self.q_s[b][t], self.kb_s[b][t], self.vb_s[b][t], self.out_s[b][t])
