@@ -17,15 +17,17 @@ namespace tc {
 #ifdef MAGE_TIMING
 __device__ unsigned long long g_stamps[128];
 __device__ __forceinline__ void stamp_at(int i) {
-    if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && i < 128) {
+    if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && i < 100) {
         unsigned long long t;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
         g_stamps[i] = t;
     }
 }
 #define MAGE_STAMP(i) stamp_at(i)
+#define MAGE_CLK(i) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) g_stamps[i] = (unsigned long long)clock64(); } while (0)
 #else
 #define MAGE_STAMP(i) ((void)0)
+#define MAGE_CLK(i) ((void)0)
 #endif
 
 constexpr int kTile = 128;                 // keys per tile
@@ -454,6 +456,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             float scale_log2, float *__restrict__ ws, __nv_bfloat16 *__restrict__ out, unsigned *status) {
     using namespace ptx;
     if (threadIdx.x == 0) MAGE_STAMP(0);
+    MAGE_CLK(126);
     if (threadIdx.x < 5) prefetch_tensormap(&maps.q + threadIdx.x);    // (kernel parameters: no need to wait for the predecessor)
     pdl_wait();                      // everything below may read what the previous kernel in the stream wrote
     pdl_launch_dependents();
@@ -1276,6 +1279,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
     __syncthreads();
     if (warp == kMmaWarp) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
     if (tid == 0) MAGE_STAMP(32);
+    MAGE_CLK(127);
 }
 
 // Merge of a reuse step that was split over n_split CTAs per KV head: one warp per query row, fixed order.
