@@ -253,6 +253,7 @@ def main():
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     if world > 1:
+        os.environ.setdefault("NCCL_DEBUG", "VERSION")      # the communicator's own line in the log says what carried the barrier
         dist.init_process_group("nccl", device_id=dev)
     mb.load()
     peaks = load_peaks()

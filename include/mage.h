@@ -233,7 +233,8 @@ mage_status mage_select_scores(const mage_kv_t *kv, const void *q, float sm_scal
  *     MAGE_ERR_WORKSPACE (and a line on stderr); nothing is launched.  As a guide, one Qwen2.5-7B-shaped layer
  *     with a 32K-token prefix needs about 18 MB; a 28-layer 128K batch does not fit.
  *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device
- *     current) and remembers it; make that first call outside any stream capture.
+ *     current) and remembers it; make that first call outside any stream capture.  The remembered address does
+ *     not survive a cudaDeviceReset of that device: do not reset a device between calls of this entry point.
  *   - The call performs no cudaMalloc / cudaFree and uses no allocating library routine.
  *   - All calls on a device share the one array, which simply keeps whatever the last call left in it.  Nothing
  *     in it has to start at zero: the kernels write every element they later read.  Two calls that can overlap
