@@ -160,3 +160,97 @@ def quest_select(Q, Kc, k, page=16):
             idx[h, : n_sel * page] = (pages[h, :n_sel, None].astype(np.int64) * page + np.arange(page)[None, :]).reshape(-1)
     return idx, n_sel * page, sc
 
+
+
+# ---------------------------------------------------------------------------------------------------------------------
+# Keys in 8 bits (the paper leaves cache compression to future work -- Limitations; this is this build's own definition
+# of the variant, stated here in full because there is no passage to restate).
+#
+#   format     e4m3: 1 sign, 4 exponent bits (bias 7), 3 mantissa bits; no infinities, largest finite value 448,
+#              smallest normal 2^-6, subnormals in steps of 2^-9
+#   scale      one per (problem, KV head): s = fl32(amax / 448), amax = largest |x| of the head's rows (1 if amax = 0)
+#   code       c = e4m3_rn_sat(fl32(x / s)): IEEE single division, then round to nearest even onto the e4m3 grid,
+#              magnitudes beyond 448 (infinities included) clamp to 448, NaN stays NaN
+#   keys       cache keys use the head's key scale s_k; the block's own keys use the same s_k (and so may clamp)
+#   queries    the G*B query rows of a KV head share s_q, taken from those rows at every call
+#   logits     s_q s_k * sum_c cq_c ck_c, everything after that as in the 16-bit path; values stay as they are
+#
+# So the variant is the unchanged method applied to the de-quantised queries and keys.  The functions below produce the
+# codes (as float64 values on the e4m3 grid) and the scales; the k8_* wrappers run the by-definition routines above head
+# by head on the codes with the head's s_q s_k folded into the softmax scale, so no value is rounded on the way in.
+# ---------------------------------------------------------------------------------------------------------------------
+E4M3_MAX = 448.0
+
+
+def e4m3_round(y):
+    """Nearest e4m3 value (ties to even, clamped to +-448, NaN kept) of each element; float64 in, float64 out."""
+    y = np.asarray(y, dtype=np.float64)
+    a = np.abs(y)
+    with np.errstate(invalid="ignore", divide="ignore"):
+        e = np.floor(np.log2(np.where((a > 0) & np.isfinite(a), a, 1.0)))
+    e = np.maximum(e, -6.0)                      # below 2^-6 the grid is the subnormal one: step 2^-9
+    step = np.exp2(e - 3.0)                      # 3 mantissa bits: 8 steps per binade
+    q = np.rint(a / step) * step                 # np.rint rounds half to even
+    q = np.where(np.isinf(a), E4M3_MAX, q)
+    q = np.minimum(q, E4M3_MAX)
+    return np.where(np.isnan(y), np.nan, np.copysign(q, y))
+
+
+def k8_scale(x):
+    """fl32(amax / 448) of an array (float32 arithmetic: the decision which code a value gets is taken in single precision)."""
+    x = np.asarray(x, dtype=np.float32)
+    amax = np.float32(np.nanmax(np.abs(x))) if x.size else np.float32(0)
+    return np.float32(1) if not amax > 0 else np.float32(amax / np.float32(448))
+
+
+def k8_codes(x, s):
+    """e4m3 codes (as float64 grid values) of x under scale s: e4m3_rn_sat(fl32(x / s))."""
+    x = np.asarray(x, dtype=np.float32)
+    with np.errstate(over="ignore", invalid="ignore"):
+        y = (x / np.float32(s)).astype(np.float32)
+    return e4m3_round(y.astype(np.float64))
+
+
+def k8_quantize_block(Q, Kc, Kb):
+    """Codes and scales of one problem.  Q [H_q,B,d], Kc [H_kv,N,d], Kb [H_kv,B,d] ->
+    (Q codes, Kc codes, Kb codes, s_q [H_kv], s_k [H_kv]); codes are float64 arrays of e4m3 grid values."""
+    Q = np.asarray(Q, dtype=np.float32); Kc = np.asarray(Kc, dtype=np.float32); Kb = np.asarray(Kb, dtype=np.float32)
+    H_q, H_kv = Q.shape[0], Kc.shape[0]
+    G = H_q // H_kv
+    s_q = np.array([k8_scale(Q[h * G:(h + 1) * G]) for h in range(H_kv)], dtype=np.float32)
+    s_k = np.array([k8_scale(Kc[h]) for h in range(H_kv)], dtype=np.float32)
+    Qc = np.concatenate([k8_codes(Q[h * G:(h + 1) * G], s_q[h]) for h in range(H_kv)], axis=0)
+    Kcc = np.stack([k8_codes(Kc[h], s_k[h]) for h in range(H_kv)])
+    Kbc = np.stack([k8_codes(Kb[h], s_k[h]) for h in range(H_kv)])
+    return Qc, Kcc, Kbc, s_q, s_k
+
+
+def _per_head(fn, Qc, s_q, s_k, scale, d, H_kv):
+    G = Qc.shape[0] // H_kv
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    return [fn(h, slice(h * G, (h + 1) * G), scale * float(s_q[h]) * float(s_k[h])) for h in range(H_kv)]
+
+
+def k8_exact_block_attn(Qc, Kcc, Vc, Kbc, Vb, s_q, s_k, scale=None, return_lse=False):
+    """exact_block_attn on 8-bit keys and queries: head by head on the codes, s_q s_k folded into the softmax scale."""
+    H_kv = Kcc.shape[0]
+    res = _per_head(lambda h, g, sc: exact_block_attn(Qc[g], Kcc[h:h + 1], Vc[h:h + 1], Kbc[h:h + 1], Vb[h:h + 1], sc, True),
+                    Qc, s_q, s_k, scale, Qc.shape[-1], H_kv)
+    O = np.concatenate([r[0] for r in res], axis=0)
+    lse = np.concatenate([r[1] for r in res], axis=0)
+    return (O, lse) if return_lse else O
+
+
+def k8_block_score(Qc, Kcc, s_q, s_k, scale=None):
+    """block_score (Eq. 4) on 8-bit keys and queries."""
+    H_kv = Kcc.shape[0]
+    res = _per_head(lambda h, g, sc: block_score(Qc[g], Kcc[h:h + 1], scale=sc), Qc, s_q, s_k, scale, Qc.shape[-1], H_kv)
+    return np.concatenate(res, axis=0)
+
+
+def k8_sparse_block_attn(Qc, Kcc, Vc, Kbc, Vb, idx, k_eff, s_q, s_k, scale=None):
+    """sparse_block_attn on 8-bit keys and queries."""
+    H_kv = Kcc.shape[0]
+    res = _per_head(lambda h, g, sc: sparse_block_attn(Qc[g], Kcc[h:h + 1], Vc[h:h + 1], Kbc[h:h + 1], Vb[h:h + 1], idx[h:h + 1], k_eff, sc),
+                    Qc, s_q, s_k, scale, Qc.shape[-1], H_kv)
+    return np.concatenate(res, axis=0)

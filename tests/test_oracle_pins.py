@@ -280,3 +280,101 @@ def test_quest_closed_forms_and_selection(oracle_mod):
     idx, k_eff, _ = oracle_mod.quest_select(Q, Kc, 64)                                   # more pages asked than exist
     assert k_eff == 48 and (idx[0, 48:] == -1).all() and idx[0, :48].tolist() == list(range(48))
 
+
+
+# ---------------------------------------------------------------------------------------------------------------------
+# 8-bit keys: the e4m3 rounding, the scales, and the wrappers that run the by-definition routines on the codes
+# ---------------------------------------------------------------------------------------------------------------------
+def _e4m3_grid():
+    """The finite e4m3 values, written out from the format: sign, 4 exponent bits (bias 7), 3 mantissa bits, 0x7f/0xff = NaN."""
+    vals = []
+    for e in range(16):
+        for m in range(8):
+            if e == 15 and m == 7:
+                continue
+            vals.append(m * 2.0 ** -9 if e == 0 else (1 + m / 8.0) * 2.0 ** (e - 7))
+    return np.array(sorted(set(vals)))
+
+
+def test_e4m3_round_grid_and_ties(oracle_mod):
+    o = oracle_mod
+    grid = _e4m3_grid()
+    assert grid.size == 127 and grid[-1] == 448.0 and grid[1] == 2.0 ** -9       # 126 positive values and zero
+    # grid values are fixed points, both signs
+    assert np.array_equal(o.e4m3_round(grid), grid) and np.array_equal(o.e4m3_round(-grid), -grid)
+    # every value lands on the grid, on a nearest neighbour, and monotonically
+    rng = np.random.default_rng(5)
+    y = np.concatenate([rng.uniform(-460, 460, 20000), rng.normal(size=20000) * 0.05, rng.normal(size=20000) * 1e-3])
+    r = o.e4m3_round(y)
+    assert np.isin(np.abs(r), grid).all()
+    clipped = np.clip(np.abs(y), 0, 448.0)
+    nearest = np.abs(grid[None, :] - clipped[:, None]).min(axis=1)
+    assert np.allclose(np.abs(np.abs(r) - clipped), nearest, rtol=0, atol=1e-15)
+    ys = np.sort(y)
+    assert (np.diff(o.e4m3_round(ys)) >= 0).all()
+    # ties go to the even mantissa: midpoints between consecutive grid values
+    mid = 0.5 * (grid[:-1] + grid[1:])
+    want = np.where((np.arange(grid.size - 1) % 2) == 0, grid[:-1], grid[1:])     # grid index = mantissa parity (zero is even)
+    assert np.array_equal(o.e4m3_round(mid), want)
+    # clamping and specials
+    assert np.array_equal(o.e4m3_round([464.0, 1e9, np.inf, -np.inf, -500.0]), [448.0, 448.0, 448.0, -448.0, -448.0])
+    assert np.isnan(o.e4m3_round([np.nan]))[0]
+    assert np.signbit(o.e4m3_round([-0.0]))[0] and o.e4m3_round([2.0 ** -11])[0] == 0.0 and o.e4m3_round([1.5 * 2.0 ** -10])[0] == 2.0 ** -9
+
+
+def test_e4m3_round_matches_library_cast(oracle_mod):
+    """torch's float -> float8_e4m3fn cast is round-to-nearest-even inside the finite range."""
+    rng = np.random.default_rng(6)
+    y = np.concatenate([rng.uniform(-448, 448, 50000), rng.normal(size=50000), rng.normal(size=50000) * 2.0 ** -7]).astype(np.float32)
+    lib = torch.from_numpy(y).to(torch.float8_e4m3fn).to(torch.float32).numpy().astype(np.float64)
+    assert np.array_equal(oracle_mod.e4m3_round(y.astype(np.float64)), lib)
+
+
+def test_k8_scale_codes_and_wrappers(oracle_mod):
+    o = oracle_mod
+    rng = np.random.default_rng(7)
+    H_kv, G, B, N, d = 2, 2, 3, 37, 16
+    bf = lambda a: torch.from_numpy(a).to(torch.bfloat16).to(torch.float32).numpy()
+    Q = bf(rng.normal(size=(H_kv * G, B, d)).astype(np.float32)); Kc = bf(rng.normal(size=(H_kv, N, d)).astype(np.float32) * 3)
+    Kb = bf(rng.normal(size=(H_kv, B, d)).astype(np.float32) * 6)                  # larger than the cache: some clamp
+    Vc = bf(rng.normal(size=(H_kv, N, d)).astype(np.float32)); Vb = bf(rng.normal(size=(H_kv, B, d)).astype(np.float32))
+    Qc, Kcc, Kbc, s_q, s_k = o.k8_quantize_block(Q, Kc, Kb)
+    grid = _e4m3_grid()
+    for h in range(H_kv):
+        amax = np.abs(Kc[h]).max()
+        assert s_k[h] == np.float32(amax / np.float32(448)) and s_k[h].dtype == np.float32
+        assert np.abs(Kcc[h]).max() == 448.0                                        # the largest element gets the largest code
+        assert np.abs(Qc[h * G:(h + 1) * G]).max() == 448.0
+        # de-quantised keys are within half a grid step (2^-4 relative for normal codes) of the originals
+        err = np.abs(Kcc[h] * float(s_k[h]) - Kc[h])
+        assert (err <= np.maximum(np.abs(Kc[h]) * 2.0 ** -4, float(s_k[h]) * 2.0 ** -10) * 1.0001).all()
+        assert np.abs(Kbc[h]).max() == 448.0 and (np.abs(Kb[h]) > amax * 1.1).any()   # block keys clamp at the cache's scale
+    assert np.isin(np.abs(Qc), grid).all() and np.isin(np.abs(Kcc), grid).all() and np.isin(np.abs(Kbc), grid).all()
+    assert o.k8_scale(np.zeros((3, 4), np.float32)) == np.float32(1) and o.k8_scale(np.zeros((0, 4), np.float32)) == np.float32(1)
+    assert np.array_equal(o.k8_codes(np.array([0.5, -0.25], np.float32), np.float32(2.0 ** -9)), [256.0, -128.0])
+    # the wrappers = the by-definition routines applied to the de-quantised tensors (written out here in float64 NumPy)
+    Qd = np.concatenate([Qc[h * G:(h + 1) * G] * float(s_q[h]) for h in range(H_kv)], axis=0)
+    Kd = Kcc * s_k.astype(np.float64)[:, None, None]; Kbd = Kbc * s_k.astype(np.float64)[:, None, None]
+    scale = 1.0 / np.sqrt(d)
+    O, lse = o.k8_exact_block_attn(Qc, Kcc, Vc, Kbc, Vb, s_q, s_k, return_lse=True)
+    sc = o.k8_block_score(Qc, Kcc, s_q, s_k)
+    for hq in range(H_kv * G):
+        h = hq // G
+        logits = np.concatenate([Qd[hq] @ Kd[h].T, Qd[hq] @ Kbd[h].T], axis=1) * scale     # [B, N + B]
+        p = np.exp(logits - logits.max(axis=1, keepdims=True)); p /= p.sum(axis=1, keepdims=True)
+        assert np.allclose(O[hq], p @ np.concatenate([Vc[h], Vb[h]], axis=0), rtol=1e-12, atol=1e-13)
+    for h in range(H_kv):
+        acc = np.zeros(N)
+        for hq in range(h * G, (h + 1) * G):
+            lg = (Qd[hq] @ Kd[h].T) * scale
+            pp = np.exp(lg - lg.max(axis=1, keepdims=True)); pp /= pp.sum(axis=1, keepdims=True)
+            acc += pp.sum(axis=0)
+        assert np.allclose(sc[h], acc / (G * B), rtol=1e-12, atol=1e-15)
+    idx, k_eff = o.topk(sc, 8)
+    Os = o.k8_sparse_block_attn(Qc, Kcc, Vc, Kbc, Vb, idx, k_eff, s_q, s_k)
+    for hq in range(H_kv * G):
+        h = hq // G
+        sel = idx[h, :k_eff]
+        logits = np.concatenate([Qd[hq] @ Kd[h][sel].T, Qd[hq] @ Kbd[h].T], axis=1) * scale
+        p = np.exp(logits - logits.max(axis=1, keepdims=True)); p /= p.sum(axis=1, keepdims=True)
+        assert np.allclose(Os[hq], p @ np.concatenate([Vc[h][sel], Vb[h]], axis=0), rtol=1e-12, atol=1e-13)
