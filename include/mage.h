@@ -292,6 +292,49 @@ mage_status mage_quest_select(const mage_kv_t *kv, const void *q, const void *pa
                               float *page_scores, int32_t *indices, int32_t *k_eff, void *workspace, size_t workspace_bytes,
                               void *stream);
 
+/*
+ * Keys and queries in 8 bits (e4m3) for Step 1 and the reuse step.  The paper leaves the compression of the cache to
+ * future work (Limitations); this variant is the library's own, defined as the unchanged method (Algorithm 1; Eq. 4)
+ * applied to de-quantised queries and keys:
+ *
+ *   scale    one per (problem, KV head): s = amax / 448 in single precision (1 when amax = 0), amax the largest |x| of the
+ *            head's rows -- the cached keys below N_p for s_k; the G*B query rows of the call for s_q, taken at every call
+ *   code     e4m3 (1 sign, 4 exponent, 3 mantissa bits; largest value 448, no infinities) of x / s: IEEE single division,
+ *            round to nearest even, magnitudes beyond 448 clamp to 448
+ *   keys     cached keys and the block's own keys use the head's s_k (block keys larger than the cache's amax clamp)
+ *   logits   s_q s_k * (code_q . code_k), accumulated in fp32 by the tensor cores; values, probabilities and outputs are
+ *            as in the 16-bit calls.  The key bytes read from the cache halve (128 instead of 256 per token and head, in
+ *            both passes of Step 1 and in the gather of the reuse step); the value bytes do not change.
+ *
+ * mage_k8_quantize_cache writes the codes of cache rows [row_begin, N_p) of every (problem, KV head):
+ *   k8_cache   device, 16-byte aligned: one byte per element, addressed exactly like kv->k_cache (same strides in
+ *              elements, same page table), so it is as large in elements as the key cache
+ *   k_scale    [P][H_kv] fp32, device.  row_begin = 0: written (from the rows below N_p); row_begin > 0: read -- rows
+ *              appended later are coded under the scale the head already has
+ *   Contiguous caches need strides that are multiples of 16 elements.
+ * mage_exact_select_k8 / mage_sparse_block_attn_k8 are mage_exact_select / mage_sparse_block_attn with the keys taken from
+ * the codes: kv->k_cache is not read (it may be NULL); kv->v_cache, q, k_blk, v_blk, the outputs and the workspace are as
+ * there.  Each call first codes its queries and block keys into k8->scratch (one small kernel).
+ *   k8->scratch  device, 256-byte aligned, at least mage_k8_scratch_bytes(kv); contents are per call
+ * Not available with MAGE_FLAG_SIMT_KERNELS, and the reuse step needs a cache that is one list of rows with a single pitch
+ * (every paged pool; contiguous layouts whose head and problem strides are multiples of the row stride): otherwise
+ * MAGE_ERR_UNSUPPORTED.  Errors as the other calls; nothing is launched unless MAGE_OK.
+ */
+typedef struct mage_k8 {
+    const void *k8_cache;  /* device: e4m3 codes of the keys                                  */
+    const float *k_scale;  /* device [P][H_kv]: de-quantisation scale of each head's keys      */
+    void *scratch;         /* device: codes of the call's queries and block keys, s_q s_k     */
+} mage_k8_t;
+size_t mage_k8_scratch_bytes(const mage_kv_t *kv);
+mage_status mage_k8_quantize_cache(const mage_kv_t *kv, int32_t row_begin, void *k8_cache, float *k_scale, uint32_t *dev_status,
+                                   void *stream);
+mage_status mage_exact_select_k8(const mage_kv_t *kv, const mage_k8_t *k8, const void *q, const void *k_blk, const void *v_blk,
+                                 float sm_scale, void *out, float *scores, void *workspace, size_t workspace_bytes,
+                                 uint32_t *dev_status, void *stream);
+mage_status mage_sparse_block_attn_k8(const mage_kv_t *kv, const mage_k8_t *k8, const void *q, const void *k_blk, const void *v_blk,
+                                      const int32_t *indices, const int32_t *k_eff, int32_t k, float sm_scale, void *out,
+                                      void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream);
+
 /* Static, human-readable name of a status code. */
 const char *mage_status_string(mage_status s);
 

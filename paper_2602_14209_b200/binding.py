@@ -28,6 +28,10 @@ class MageError(RuntimeError):
         super().__init__(f"{where}: {status_string(code)} ({code})")
 
 
+class mage_k8_t(ctypes.Structure):
+    _fields_ = [("k8_cache", ctypes.c_void_p), ("k_scale", ctypes.c_void_p), ("scratch", ctypes.c_void_p)]
+
+
 class mage_kv_t(ctypes.Structure):
     _fields_ = [
         ("P", ctypes.c_int32), ("H_q", ctypes.c_int32), ("H_kv", ctypes.c_int32), ("d", ctypes.c_int32),
@@ -40,6 +44,7 @@ class mage_kv_t(ctypes.Structure):
 
 
 EXPORTS = ("mage_pruned_workspace_bytes", "mage_exact_select_pruned", "mage_quest_workspace_bytes", "mage_quest_build", "mage_quest_select", "mage_append_block", "mage_workspace_bytes", "mage_exact_select", "mage_exact_select_events", "mage_exact_select_static", "mage_exact_attn", "mage_select_scores", "mage_topk", "mage_sparse_block_attn",
+           "mage_k8_scratch_bytes", "mage_k8_quantize_cache", "mage_exact_select_k8", "mage_sparse_block_attn_k8",
            "mage_status_string", "mage_launch_count")
 
 
@@ -81,6 +86,16 @@ def load():
     lib.mage_quest_build.argtypes = [ctypes.POINTER(mage_kv_t), vp, vp, vp, vp]
     lib.mage_quest_select.restype = ctypes.c_int
     lib.mage_quest_select.argtypes = [ctypes.POINTER(mage_kv_t), vp, vp, vp, i32, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.mage_k8_scratch_bytes.restype = ctypes.c_size_t
+    lib.mage_k8_scratch_bytes.argtypes = [ctypes.POINTER(mage_kv_t)]
+    lib.mage_k8_quantize_cache.restype = ctypes.c_int
+    lib.mage_k8_quantize_cache.argtypes = [ctypes.POINTER(mage_kv_t), i32, vp, vp, vp, vp]
+    lib.mage_exact_select_k8.restype = ctypes.c_int
+    lib.mage_exact_select_k8.argtypes = [ctypes.POINTER(mage_kv_t), ctypes.POINTER(mage_k8_t), vp, vp, vp, ctypes.c_float, vp, vp, vp,
+                                         ctypes.c_size_t, vp, vp]
+    lib.mage_sparse_block_attn_k8.restype = ctypes.c_int
+    lib.mage_sparse_block_attn_k8.argtypes = [ctypes.POINTER(mage_kv_t), ctypes.POINTER(mage_k8_t), vp, vp, vp, vp, vp, i32, ctypes.c_float,
+                                              vp, vp, ctypes.c_size_t, vp, vp]
     lib.mage_status_string.restype = ctypes.c_char_p
     lib.mage_status_string.argtypes = [ctypes.c_int]
     lib.mage_launch_count.restype = u64
@@ -225,6 +240,48 @@ def mage_sparse_block_attn(kv: KVCache, q, k_blk, v_blk, indices, k_eff, k: int,
                                        _ptr(dev_status), _stream(stream))
     if rc != MAGE_OK:
         raise MageError(rc, "mage_sparse_block_attn")
+
+
+class K8Keys:
+    """The keys of a cache as e4m3 codes (``mage_k8_t``): ``codes`` is a uint8 tensor shaped and strided like ``kv.k``,
+    ``k_scale`` is [P, H_kv] fp32, ``scratch`` the per-call buffer.  ``quantize`` fills codes (and, from row 0, the scales)."""
+
+    def __init__(self, kv: KVCache):
+        self.kv = kv
+        self.codes = torch.empty_strided(kv.k.shape, kv.k.stride(), dtype=torch.uint8, device=kv.device)
+        self.k_scale = torch.empty(kv.P, kv.H_kv, dtype=torch.float32, device=kv.device)
+        n = int(load().mage_k8_scratch_bytes(ctypes.byref(kv.c)))
+        if n == 0:
+            raise MageError(-1, "mage_k8_scratch_bytes")
+        self.scratch = torch.empty(n, dtype=torch.uint8, device=kv.device)
+        self.c = mage_k8_t(self.codes.data_ptr(), self.k_scale.data_ptr(), self.scratch.data_ptr())
+
+    def quantize(self, row_begin: int = 0, dev_status=None, stream=None):
+        rc = load().mage_k8_quantize_cache(ctypes.byref(self.kv.c), int(row_begin), _ptr(self.codes), _ptr(self.k_scale), _ptr(dev_status),
+                                           _stream(stream))
+        if rc != MAGE_OK:
+            raise MageError(rc, "mage_k8_quantize_cache")
+        return self
+
+
+def mage_exact_select_k8(kv: KVCache, k8: K8Keys, q, k_blk, v_blk, sm_scale: float, out, scores, workspace, dev_status=None, stream=None):
+    """mage_exact_select with the keys (and queries) in 8 bits (see mage.h)."""
+    rc = load().mage_exact_select_k8(ctypes.byref(kv.c), ctypes.byref(k8.c), _ptr(q), _ptr(k_blk), _ptr(v_blk), float(sm_scale), _ptr(out),
+                                     _ptr(scores), _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(dev_status),
+                                     _stream(stream))
+    if rc != MAGE_OK:
+        raise MageError(rc, "mage_exact_select_k8")
+
+
+def mage_sparse_block_attn_k8(kv: KVCache, k8: K8Keys, q, k_blk, v_blk, indices, k_eff, k: int, sm_scale: float, out, workspace=None,
+                              dev_status=None, stream=None):
+    """mage_sparse_block_attn with the keys (and queries) in 8 bits (see mage.h)."""
+    rc = load().mage_sparse_block_attn_k8(ctypes.byref(kv.c), ctypes.byref(k8.c), _ptr(q), _ptr(k_blk), _ptr(v_blk), _ptr(indices),
+                                          _ptr(k_eff), int(k), float(sm_scale), _ptr(out), _ptr(workspace),
+                                          workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                          _ptr(dev_status), _stream(stream))
+    if rc != MAGE_OK:
+        raise MageError(rc, "mage_sparse_block_attn_k8")
 
 
 def mage_append_block(kv: KVCache, k_blk, v_blk, seq_lens, dev_status=None, stream=None):

@@ -6,6 +6,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "k8.cuh"
 #include "prune.cuh"
 #include "quest.cuh"
 #include "simt_kernels.cuh"
@@ -151,7 +152,7 @@ static mage_status opt_in_smem(K kernel, size_t bytes) { return opt_in_smem_impl
 
 // Why the tensor-core kernels cannot take this description, or MAGE_OK.  There is one production path; the portable
 // CUDA-core kernels run only when the caller asks for them with MAGE_FLAG_SIMT_KERNELS, never as a silent substitute.
-static mage_status tc_supported(const mage_kv_t *kv) {
+static mage_status tc_supported(const mage_kv_t *kv) {   // (8-bit keys: the caller's copy of kv carries the codes as k_cache)
     if (kv->page_size != 0 && kv->page_size % 64 != 0) return MAGE_ERR_UNSUPPORTED;        // a 64-key TMA box must lie inside one page
     if (kv->N_max > 0 && ((reinterpret_cast<uintptr_t>(kv->k_cache) | reinterpret_cast<uintptr_t>(kv->v_cache)) & 15)) return MAGE_ERR_UNSUPPORTED;
     if (tc::encode_fn() == nullptr) return MAGE_ERR_CUDA;
@@ -161,11 +162,12 @@ static mage_status tc_supported(const mage_kv_t *kv) {
 // The block-score pass (Eq. 4) over all key tiles, or over the tiles of `list`: grid_x CTAs of tiles_per_cta tiles per head.
 static mage_status launch_score_pass(const KvView &view, const Plan &plan, const CUtensorMap &map_q_rows, const CUtensorMap &map_k,
                                      int grid_x, int tiles_per_cta, float scale_log2, const float *ws, float *scores,
-                                     unsigned *dev_status, cudaStream_t st, const tc::ScoreTileList &list) {
+                                     unsigned *dev_status, cudaStream_t st, const tc::ScoreTileList &list,
+                                     const float *qk_scale = nullptr) {
     dim3 sgrid(grid_x, view.P * view.H_kv, 1);
     for (int r0 = 0; r0 < view.M; r0 += 256) {
-        launch_pdl(tc::score_kernel, sgrid, dim3(tc::kScoreThreads), tc::kScoreSmemBytes, st, map_q_rows, map_k, view, plan, r0, std::min(256, view.M - r0),
-                   tiles_per_cta, scale_log2, ws, scores, (int)(r0 > 0), dev_status, list);
+        launch_pdl(qk_scale ? tc::score_kernel<true> : tc::score_kernel<false>, sgrid, dim3(tc::kScoreThreads), tc::kScoreSmemBytes, st, map_q_rows, map_k, view, plan, r0, std::min(256, view.M - r0),
+                   tiles_per_cta, scale_log2, ws, scores, (int)(r0 > 0), dev_status, list, qk_scale);
         if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
     }
     return MAGE_OK;
@@ -175,13 +177,35 @@ static mage_status launch_score_pass(const KvView &view, const Plan &plan, const
 // the block-score pass.  scores_only: the select stream's own computation (Algorithm 1: A = softmax(Q K^T / sqrt d) over
 // the prefix, then the mean over the block's rows) without the attention output: pass A keeps only the rows' maxima and
 // sums (no V, no P V, no block keys), the merge emits only the log-sum-exp, pass B is unchanged; k_blk, v_blk, out unused.
+// 8-bit keys: the codes of the cache with their scales (caller's), and the per-call scratch of the codes of the queries and
+// the block's keys with the heads' factors s_q s_k.
+struct K8 {
+    const uint8_t *k8;
+    const float *k_scale;
+    uint8_t *q8, *kb8;
+    float *qk_scale;
+};
+static size_t k8_scratch_layout(const mage_kv_t *kv, size_t *off_kb8, size_t *off_qk) {
+    const size_t q8 = align_up((size_t)kv->P * kv->H_q * kv->B * kD, 256), kb8 = align_up((size_t)kv->P * kv->H_kv * kv->B * kD, 256);
+    if (off_kb8) *off_kb8 = q8;
+    if (off_qk) *off_qk = q8 + kb8;
+    return q8 + kb8 + align_up((size_t)kv->P * kv->H_kv * sizeof(float), 256);
+}
+// Codes of the call's queries and block keys (one small kernel in front of the pass that uses them).
+static mage_status launch_block_codes(const KvView &view, const K8 &k8, const __nv_bfloat16 *q, const __nv_bfloat16 *k_blk, cudaStream_t st) {
+    k8::block_code_kernel<<<view.P * view.H_kv, 256, 0, st>>>(view, q, k_blk, k8.k_scale, k8.q8, k8.kb8, k8.qk_scale);
+    return launch_check();
+}
+
 static mage_status launch_exact_select(const mage_kv_t *kv, const KvView &view, const Plan &plan, const __nv_bfloat16 *q,
                                        const __nv_bfloat16 *k_blk, const __nv_bfloat16 *v_blk, float sm_scale,
                                        __nv_bfloat16 *out, float *scores, float *ws, unsigned *dev_status, cudaStream_t st,
-                                       cudaEvent_t *ev, bool scores_only = false, float2 *rowsum = nullptr, int rowsum_tiles = 0) {
+                                       cudaEvent_t *ev, bool scores_only = false, float2 *rowsum = nullptr, int rowsum_tiles = 0,
+                                       const K8 *k8 = nullptr) {
     const float scale_log2 = sm_scale * kLog2e;
     const int heads = kv->P * kv->H_kv, rows_total = heads * view.M;
     const int n_items = plan.n_chunks + (scores_only ? 0 : 1);
+    if (k8 && ((kv->flags & MAGE_FLAG_SIMT_KERNELS) || scores_only)) return MAGE_ERR_UNSUPPORTED;
     if (kv->flags & MAGE_FLAG_SIMT_KERNELS) {
         using namespace simt;
         auto kern = attn_kernel<Mode::kExactPartial>;
@@ -207,15 +231,19 @@ static mage_status launch_exact_select(const mage_kv_t *kv, const KvView &view, 
     // every tensor map is encoded before the first launch: a description that cannot be encoded launches nothing
     tc::AttnMaps maps;
     CUtensorMap map_q_rows, map_k_score;
-    auto kern_tc = tc::attn_kernel<false>;
-    bool maps_ok = tc::make_group_rows_map(&maps.q, q, heads, view.M);
-    if (maps_ok && kv->N_max > 0) maps_ok = tc::make_cache_map(&maps.k, kv, kv->k_cache);
+    auto kern_tc = k8 ? tc::attn_kernel<false, true> : tc::attn_kernel<false, false>;
+    const int eb = k8 ? 1 : 2;                             // bytes per query / key element
+    const void *q_src = k8 ? (const void *)k8->q8 : (const void *)q, *kc_src = k8 ? (const void *)k8->k8 : kv->k_cache;
+    const void *kb_src = k8 ? (const void *)k8->kb8 : (const void *)k_blk;
+    bool maps_ok = tc::make_group_rows_map(&maps.q, q_src, heads, view.M, eb);
+    if (maps_ok && kv->N_max > 0) maps_ok = tc::make_cache_map(&maps.k, kv, kc_src, eb);
     else maps.k = maps.q;                                  // no prefix: never used
+    if (k8) maps.qk_scale = k8->qk_scale;
     if (maps_ok && scores_only) {
         maps.v = maps.kb = maps.vb = maps.k;              // never used in this mode
         maps.lse_only = 1;
     } else if (maps_ok) {
-        maps_ok = tc::make_rows_map(&maps.kb, k_blk, (long long)heads * kv->B) && tc::make_rows_map(&maps.vb, v_blk, (long long)heads * kv->B);
+        maps_ok = tc::make_rows_map(&maps.kb, kb_src, (long long)heads * kv->B, eb) && tc::make_rows_map(&maps.vb, v_blk, (long long)heads * kv->B);
         if (maps_ok && kv->N_max > 0) maps_ok = tc::make_cache_map(&maps.v, kv, kv->v_cache);
         else maps.v = maps.q;
     }
@@ -223,10 +251,13 @@ static mage_status launch_exact_select(const mage_kv_t *kv, const KvView &view, 
     maps.rowsum = rowsum;
     maps.rowsum_tiles = rowsum_tiles;
     const bool want_scores = scores && kv->N_max > 0;
-    if (maps_ok && want_scores) maps_ok = tc::make_rows_map(&map_q_rows, q, (long long)kv->P * kv->H_q * kv->B) && tc::make_cache_map(&map_k_score, kv, kv->k_cache);
+    if (maps_ok && want_scores) maps_ok = tc::make_rows_map(&map_q_rows, q_src, (long long)kv->P * kv->H_q * kv->B, eb) && tc::make_cache_map(&map_k_score, kv, kc_src, eb);
     if (!maps_ok) return MAGE_ERR_UNSUPPORTED;
-    if (opt_in_smem(kern_tc, tc::kAttnSmemBytesDense) != MAGE_OK || opt_in_smem(tc::score_kernel, tc::kScoreSmemBytes) != MAGE_OK) return MAGE_ERR_CUDA;
+    if (opt_in_smem(kern_tc, tc::kAttnSmemBytesDense) != MAGE_OK || opt_in_smem(tc::score_kernel<false>, tc::kScoreSmemBytes) != MAGE_OK ||
+        opt_in_smem(tc::score_kernel<true>, tc::kScoreSmemBytes) != MAGE_OK)
+        return MAGE_ERR_CUDA;
     if (ev) cudaEventRecord(ev[0], st);
+    if (k8 && launch_block_codes(view, *k8, q, k_blk, st) != MAGE_OK) return MAGE_ERR_CUDA;
     if (n_items > 0) {
         launch_pdl(kern_tc, dim3(n_items, (view.M + 255) / 256, heads), dim3(320), tc::kAttnSmemBytesDense, st, maps, view, plan, k_blk, v_blk, (const int *)nullptr,
                    (const int *)nullptr, 0, scale_log2, ws, (__nv_bfloat16 *)nullptr, dev_status);
@@ -239,7 +270,8 @@ static mage_status launch_exact_select(const mage_kv_t *kv, const KvView &view, 
     if (want_scores) {
         const int tpc = tc::tiles_per_cta_for(heads, kv->N_max, kv->page_size != 0);
         const int tiles_head = (kv->N_max + tc::kTile - 1) / tc::kTile;
-        if (launch_score_pass(view, plan, map_q_rows, map_k_score, (tiles_head + tpc - 1) / tpc, tpc, scale_log2, ws, scores, dev_status, st, tc::ScoreTileList()) != MAGE_OK)
+        if (launch_score_pass(view, plan, map_q_rows, map_k_score, (tiles_head + tpc - 1) / tpc, tpc, scale_log2, ws, scores, dev_status, st, tc::ScoreTileList(),
+                              k8 ? k8->qk_scale : nullptr) != MAGE_OK)
             return MAGE_ERR_CUDA;
     }
     if (ev) cudaEventRecord(ev[3], st);
@@ -250,8 +282,9 @@ static mage_status launch_exact_select(const mage_kv_t *kv, const KvView &view, 
 static mage_status launch_sparse_step(const mage_kv_t *kv, const KvView &view, const Plan &plan, const __nv_bfloat16 *q,
                                       const __nv_bfloat16 *k_blk, const __nv_bfloat16 *v_blk, const int *indices,
                                       const int *k_eff, int k, float sm_scale, __nv_bfloat16 *out, float *ws, bool ws_ok,
-                                      unsigned *dev_status, cudaStream_t st) {
+                                      unsigned *dev_status, cudaStream_t st, const K8 *k8 = nullptr) {
     const int heads = kv->P * kv->H_kv;
+    if (k8 && (kv->flags & MAGE_FLAG_SIMT_KERNELS)) return MAGE_ERR_UNSUPPORTED;
     if (kv->flags & MAGE_FLAG_SIMT_KERNELS) {
         using namespace simt;
         auto kern = attn_kernel<Mode::kSparseFinal>;
@@ -261,22 +294,33 @@ static mage_status launch_sparse_step(const mage_kv_t *kv, const KvView &view, c
     }
     if (tc::encode_fn() == nullptr) return MAGE_ERR_CUDA;
     tc::AttnMaps maps;
-    auto kern_tc = tc::attn_kernel<true>;
-    if (!tc::make_group_rows_map(&maps.q, q, heads, view.M)) return MAGE_ERR_UNSUPPORTED;
+    auto kern_tc = k8 ? tc::attn_kernel<true, true> : tc::attn_kernel<true, false>;
+    const int eb = k8 ? 1 : 2;
+    const void *q_src = k8 ? (const void *)k8->q8 : (const void *)q, *kc_src = k8 ? (const void *)k8->k8 : kv->k_cache;
+    const void *kb_src = k8 ? (const void *)k8->kb8 : (const void *)k_blk;
+    if (!tc::make_group_rows_map(&maps.q, q_src, heads, view.M, eb)) return MAGE_ERR_UNSUPPORTED;
+    if (k8) maps.qk_scale = k8->qk_scale;
     maps.k = maps.v = maps.kb = maps.vb = maps.q;         // placeholders unless the TMA row gather below applies
     // Two gathers inside the one kernel: single 256-byte rows by TMA when the cache is one list of rows with a single pitch
     // (every paged pool; contiguous layouts whose head and problem strides are multiples of the row stride), otherwise
     // 16-byte cp.async, which addresses rows through 32-bit offsets in 16-byte units.
     long long c_rows = 0, c_pitch = 0;
     const long long b_rows = (long long)heads * kv->B;
-    const bool aligned = !((reinterpret_cast<uintptr_t>(kv->k_cache) | reinterpret_cast<uintptr_t>(kv->v_cache) | reinterpret_cast<uintptr_t>(k_blk) |
+    const bool aligned = !((reinterpret_cast<uintptr_t>(kc_src) | reinterpret_cast<uintptr_t>(kv->v_cache) | reinterpret_cast<uintptr_t>(kb_src) |
                             reinterpret_cast<uintptr_t>(v_blk)) & 15);
-    if (kv->N_max > 0 && aligned && tc::cache_as_rows(kv, &c_rows, &c_pitch) && tc::make_row_gather_map(&maps.k, kv->k_cache, c_rows, c_pitch) &&
-        tc::make_row_gather_map(&maps.v, kv->v_cache, c_rows, c_pitch) && tc::make_row_gather_map(&maps.kb, k_blk, b_rows, kD) &&
+    if (kv->N_max > 0 && aligned && tc::cache_as_rows(kv, &c_rows, &c_pitch) && tc::make_row_gather_map(&maps.k, kc_src, c_rows, c_pitch, eb) &&
+        tc::make_row_gather_map(&maps.v, kv->v_cache, c_rows, c_pitch) && tc::make_row_gather_map(&maps.kb, kb_src, b_rows, kD, eb) &&
         tc::make_row_gather_map(&maps.vb, v_blk, b_rows, kD)) {
         maps.gather_rows = (int)c_rows;
         maps.gather_blk_rows = (int)b_rows;
         maps.gather_pitch = (int)c_pitch;
+    } else if (k8) {                                       // 8-bit keys are gathered by TMA only (a cache with one row pitch)
+        if (kv->N_max != 0 || !aligned || !tc::make_row_gather_map(&maps.kb, kb_src, b_rows, kD, eb) || !tc::make_row_gather_map(&maps.vb, v_blk, b_rows, kD))
+            return MAGE_ERR_UNSUPPORTED;
+        maps.k = maps.kb;                                  // no prefix: every request names the block's rows
+        maps.v = maps.vb;
+        maps.gather_rows = maps.gather_blk_rows = (int)b_rows;
+        maps.gather_pitch = kD;
     } else {
         if (!aligned) return MAGE_ERR_UNSUPPORTED;        // cp.async moves 16-byte pieces
         const long long last = kv->page_size ? (long long)kv->num_pages * kv->H_kv * kv->page_size * kD
@@ -294,6 +338,7 @@ static mage_status launch_sparse_step(const mage_kv_t *kv, const KvView &view, c
         if (n_split > plan.sparse_split_max) n_split = plan.sparse_split_max;
         if (n_split < 1) n_split = 1;
     }
+    if (k8 && launch_block_codes(view, *k8, q, k_blk, st) != MAGE_OK) return MAGE_ERR_CUDA;
     launch_pdl(kern_tc, dim3(n_split, n_rg, heads), dim3(tc::kSparseThreads), tc::kAttnSmemBytesSparse, st, maps, view, plan, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, ws, out, dev_status);
     if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
     if (n_split > 1) {
@@ -406,6 +451,95 @@ mage_status mage_sparse_block_attn(const mage_kv_t *kv, const void *q, const voi
     return launch_sparse_step(kv, view, plan, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_blk),
                        static_cast<const __nv_bfloat16 *>(v_blk), indices, k_eff, k, sm_scale, static_cast<__nv_bfloat16 *>(out),
                        static_cast<float *>(workspace), ws_ok, dev_status, static_cast<cudaStream_t>(stream));
+}
+
+// ---- 8-bit keys
+static bool valid_k8(const mage_kv_t *kv, const mage_k8_t *k8, K8 *out) {
+    if (!k8 || !k8->scratch || (reinterpret_cast<uintptr_t>(k8->scratch) & 255)) return false;
+    if (kv->N_max > 0 && (!k8->k8_cache || !k8->k_scale)) return false;
+    if (!k8->k_scale) return false;
+    size_t off_kb8 = 0, off_qk = 0;
+    k8_scratch_layout(kv, &off_kb8, &off_qk);
+    uint8_t *base = static_cast<uint8_t *>(k8->scratch);
+    out->k8 = static_cast<const uint8_t *>(k8->k8_cache);
+    out->k_scale = k8->k_scale;
+    out->q8 = base;
+    out->kb8 = base + off_kb8;
+    out->qk_scale = reinterpret_cast<float *>(base + off_qk);
+    return true;
+}
+
+size_t mage_k8_scratch_bytes(const mage_kv_t *kv) {
+    if (!valid_kv(kv, nullptr)) return 0;
+    return k8_scratch_layout(kv, nullptr, nullptr);
+}
+
+mage_status mage_k8_quantize_cache(const mage_kv_t *kv, int32_t row_begin, void *k8_cache, float *k_scale, uint32_t *dev_status, void *stream) {
+    mage_status why = MAGE_OK;
+    if (!valid_kv(kv, &why)) return why;
+    if (!k_scale || row_begin < 0 || (kv->N_max > 0 && !k8_cache)) return MAGE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(k8_cache) | reinterpret_cast<uintptr_t>(kv->k_cache)) & 15) return MAGE_ERR_UNSUPPORTED;
+    if (kv->page_size == 0 && (kv->stride_n % 16 || kv->stride_h % 16 || kv->stride_p % 16)) return MAGE_ERR_UNSUPPORTED;   // 16 codes per store
+    const KvView view = make_view(kv);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int heads = kv->P * kv->H_kv;
+    const int rows = kv->N_max - row_begin;
+    if (row_begin == 0) {                                  // the scales are taken from the rows that are there now
+        if (cudaMemsetAsync(k_scale, 0, (size_t)heads * sizeof(float), st) != cudaSuccess) return MAGE_ERR_CUDA;
+        if (rows > 0) {
+            k8::cache_amax_kernel<<<dim3((rows + k8::kRowsPerCta - 1) / k8::kRowsPerCta, heads), 256, 0, st>>>(view, 0, reinterpret_cast<unsigned *>(k_scale), dev_status);
+            if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+        }
+        k8::amax_to_scale_kernel<<<(heads + 127) / 128, 128, 0, st>>>(k_scale, heads);
+        if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    }
+    if (rows > 0) {
+        k8::cache_code_kernel<<<dim3((rows + k8::kRowsPerCta - 1) / k8::kRowsPerCta, heads), 256, 0, st>>>(view, row_begin, k_scale, static_cast<uint8_t *>(k8_cache), dev_status);
+        if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
+    }
+    return MAGE_OK;
+}
+
+mage_status mage_exact_select_k8(const mage_kv_t *kv, const mage_k8_t *k8, const void *q, const void *k_blk, const void *v_blk,
+                                 float sm_scale, void *out, float *scores, void *workspace, size_t workspace_bytes,
+                                 uint32_t *dev_status, void *stream) {
+    if (!kv || !k8) return MAGE_ERR_INVALID_ARG;
+    mage_kv_t kvc = *kv;
+    kvc.k_cache = k8->k8_cache;                            // the 16-bit keys are not read
+    mage_status why = MAGE_OK;
+    if (!valid_kv(&kvc, &why)) return why;
+    K8 a;
+    if (!valid_k8(&kvc, k8, &a)) return MAGE_ERR_INVALID_ARG;
+    if (!q || !k_blk || !v_blk || !out || !workspace || (kvc.N_max > 0 && !scores)) return MAGE_ERR_INVALID_ARG;
+    if (!(sm_scale > 0.f) || (reinterpret_cast<uintptr_t>(workspace) & 255)) return MAGE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k_blk)) & 15) return MAGE_ERR_UNSUPPORTED;
+    const Plan plan = make_plan(&kvc);
+    if (workspace_bytes < plan.exact_bytes) return MAGE_ERR_WORKSPACE;
+    const KvView view = make_view(&kvc);
+    return launch_exact_select(&kvc, view, plan, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_blk),
+                               static_cast<const __nv_bfloat16 *>(v_blk), sm_scale, static_cast<__nv_bfloat16 *>(out), scores,
+                               static_cast<float *>(workspace), dev_status, static_cast<cudaStream_t>(stream), nullptr, false, nullptr, 0, &a);
+}
+
+mage_status mage_sparse_block_attn_k8(const mage_kv_t *kv, const mage_k8_t *k8, const void *q, const void *k_blk, const void *v_blk,
+                                      const int32_t *indices, const int32_t *k_eff, int32_t k, float sm_scale, void *out,
+                                      void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream) {
+    if (!kv || !k8) return MAGE_ERR_INVALID_ARG;
+    mage_kv_t kvc = *kv;
+    kvc.k_cache = k8->k8_cache;
+    mage_status why = MAGE_OK;
+    if (!valid_kv(&kvc, &why)) return why;
+    K8 a;
+    if (!valid_k8(&kvc, k8, &a)) return MAGE_ERR_INVALID_ARG;
+    if (!q || !k_blk || !v_blk || !out || !indices || !k_eff || k < 1) return MAGE_ERR_INVALID_ARG;
+    if (!(sm_scale > 0.f)) return MAGE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k_blk)) & 15) return MAGE_ERR_UNSUPPORTED;
+    const Plan plan = make_plan(&kvc, k);
+    const KvView view = make_view(&kvc);
+    const bool ws_ok = workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255) && workspace_bytes >= plan.total_bytes;
+    return launch_sparse_step(&kvc, view, plan, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_blk),
+                              static_cast<const __nv_bfloat16 *>(v_blk), indices, k_eff, k, sm_scale, static_cast<__nv_bfloat16 *>(out),
+                              static_cast<float *>(workspace), ws_ok, dev_status, static_cast<cudaStream_t>(stream), &a);
 }
 
 mage_status mage_append_block(const mage_kv_t *kv, const void *k_blk, const void *v_blk, int32_t *seq_lens, uint32_t *dev_status,

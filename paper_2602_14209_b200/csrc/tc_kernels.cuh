@@ -110,14 +110,19 @@ constexpr int kScoreProducerWarp = kScoreWgs * 4, kScoreMmaWarp = kScoreWgs * 4 
 constexpr int kScoreQBytes = 2 * 256 * 128;           // up to 256 query rows, two d-halves
 constexpr size_t kScoreSmemBytes = 1024 + kScoreQBytes + kScoreStages * kTileBytes + (256 + 2 * 128) * sizeof(float) + 320;
 
+// K8: queries and keys arrive as e4m3 codes (rows of 128 bytes, one 128-byte swizzle atom per row, so a tile is one
+// d-"half" of the 16-bit layout), the products run on the 8-bit MMA kind, and the head's factor s_q s_k (qk_scale) goes
+// into the exponent's scale.  Everything after the logits is the same code.
+template <bool K8>
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, KvView kv, Plan plan,
              int row_begin, int rows, int tiles_per_cta, float scale_log2, const float *__restrict__ ws,
-             float *__restrict__ scores, int accumulate, unsigned *status, ScoreTileList list) {
+             float *__restrict__ scores, int accumulate, unsigned *status, ScoreTileList list, const float *__restrict__ qk_scale) {
     using namespace ptx;
     pdl_wait();
     pdl_launch_dependents();
     const int z = blockIdx.y, p = z / kv.H_kv, h = z % kv.H_kv;
+    if (K8) scale_log2 *= qk_scale[z];
     const int N = seq_len_of(kv, p);
     // list mode (pruned selection): the CTA walks entries [tile0, tile0 + n_my) of this head's ascending list of tile numbers
     const int *my_list = list.tiles ? list.tiles + (size_t)z * list.stride : nullptr;
@@ -175,8 +180,8 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
             prefetch_tensormap(&map_q);
             prefetch_tensormap(&map_k);
             const int q_row0 = (p * kv.H_q + h * kv.G) * kv.B + row_begin;
-            mbar_arrive_expect_tx(bar(Q_FULL), 2 * rows64 * 128);
-            for (int dh = 0; dh < 2; ++dh)
+            mbar_arrive_expect_tx(bar(Q_FULL), (K8 ? 1 : 2) * rows64 * 128);
+            for (int dh = 0; dh < (K8 ? 1 : 2); ++dh)
                 for (int rb = 0; rb < rows64 / 64; ++rb)
                     tma_load_2d(smem_u32(q_s + dh * (kScoreQBytes / 2) + rb * kBoxBytes), &map_q, bar(Q_FULL), dh * 64, q_row0 + rb * 64);
             const uint64_t pol_k = l2_policy_evict_first();       // last use of these K lines
@@ -205,9 +210,9 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                 } else {
                     for (int kh = 0; kh < 2; ++kh) cache_box_coords(kv, p, h, j0 + kh * 64, N, c1[kh], c2[kh], c3[kh], nullptr);
                 }
-                mbar_arrive_expect_tx(bar(FULL + slot), kTileBytes);
+                mbar_arrive_expect_tx(bar(FULL + slot), K8 ? kHalfBytes : kTileBytes);
                 for (int kh = 0; kh < 2; ++kh)
-                    for (int dh = 0; dh < 2; ++dh)
+                    for (int dh = 0; dh < (K8 ? 1 : 2); ++dh)
                         tma_load_4d_hint(smem_u32(k_s + slot * kTileBytes + dh * kHalfBytes + kh * kBoxBytes), &map_k, bar(FULL + slot), dh * 64, c1[kh], c2[kh], c3[kh], pol_k);
                 issued = i + 1;
             }
@@ -220,8 +225,8 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
         }
     } else if (warp == kScoreMmaWarp) {
         if (lane == 0) {
-            const uint32_t idesc_lo = idesc_bf16_f32((rows_lo + 15) & ~15, false, false);
-            const uint32_t idesc_hi = idesc_bf16_f32(max(16, (rows_hi + 15) & ~15), false, false);
+            const uint32_t idesc_lo = K8 ? idesc_e4m3_f32((rows_lo + 15) & ~15) : idesc_bf16_f32((rows_lo + 15) & ~15, false, false);
+            const uint32_t idesc_hi = K8 ? idesc_e4m3_f32(max(16, (rows_hi + 15) & ~15)) : idesc_bf16_f32(max(16, (rows_hi + 15) & ~15), false, false);
             bool ok = mbar_wait(bar(Q_FULL), 0, abort_s, status);
             for (int i = 0; ok && i < n_my; ++i) {
                 const int slot = i % kScoreStages, su = i / kScoreStages;
@@ -231,12 +236,21 @@ score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                     const int buf = quad ? (i & 3) : (i & 1) * 2 + rh, use = quad ? i >> 2 : i >> 1;     // buffer = warpgroup that consumes it
                     if (!mbar_wait(bar(T_EMPTY + buf), (use & 1) ^ 1, abort_s, status)) { ok = false; break; }
                     tc_fence_after_sync();
+                    if (K8) {                                  // 32 one-byte elements of d per step: the whole row is one atom
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                        const uint64_t a = smem_desc_sw128(k_addr + off, 16, 1024);
-                        const uint64_t b = smem_desc_sw128(q_addr + (ks >> 2) * (kScoreQBytes / 2) + (ks & 3) * 32 + rh * rows_lo * 128, 16, 1024);
-                        umma_ss(tmem_base + buf * 128, a, b, rh ? idesc_hi : idesc_lo, ks > 0);
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint64_t a = smem_desc_sw128(k_addr + ks * 32, 16, 1024);
+                            const uint64_t b = smem_desc_sw128(q_addr + ks * 32 + rh * rows_lo * 128, 16, 1024);
+                            umma_ss_f8(tmem_base + buf * 128, a, b, rh ? idesc_hi : idesc_lo, ks > 0);
+                        }
+                    } else {
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks) {
+                            const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+                            const uint64_t a = smem_desc_sw128(k_addr + off, 16, 1024);
+                            const uint64_t b = smem_desc_sw128(q_addr + (ks >> 2) * (kScoreQBytes / 2) + (ks & 3) * 32 + rh * rows_lo * 128, 16, 1024);
+                            umma_ss(tmem_base + buf * 128, a, b, rh ? idesc_hi : idesc_lo, ks > 0);
+                        }
                     }
                     umma_commit(bar(T_FULL + buf));
                 }
@@ -447,9 +461,13 @@ struct AttnMaps {
     float2 *rowsum = nullptr;
     int rowsum_tiles = 0;
     int test_stall = 0;          // MAGE_FLAG_TEST_STALL: the exact pass never requests its first key tile and waits with the short limit
+    const float *qk_scale = nullptr;   // 8-bit keys: s_q s_k per (problem, KV head); q, k, kb are then maps of e4m3 codes
 };
 
-template <bool SPARSE>
+// K8: queries and keys (cache and block) are e4m3 codes in rows of 128 bytes; a Q or K tile then fills the first d-"half"
+// of its 32 KB region, Q K^T runs on the 8-bit MMA kind in four steps of 32 elements, and the head's s_q s_k goes into the
+// softmax scale.  Values, P and P V are as in the 16-bit kernel.
+template <bool SPARSE, bool K8 = false>
 __global__ void __launch_bounds__(SPARSE ? kSparseThreads : 320, 1)
 attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const __nv_bfloat16 *__restrict__ k_blk,
             const __nv_bfloat16 *__restrict__ v_blk, const int *__restrict__ indices, const int *__restrict__ k_eff_arr, int k,
@@ -465,6 +483,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
     constexpr int kAttnSlots = SPARSE ? kAttnSlotsSparse : kAttnSlotsDense;
     const int chunk = blockIdx.x, rg = blockIdx.y, z = blockIdx.z, p = z / kv.H_kv, h = z % kv.H_kv;
     const int N = seq_len_of(kv, p);
+    if (K8) scale_log2 *= maps.qk_scale[z];
     int n_keys, n_cache, j_begin = 0, first_idx = 0;
     bool blk_chunk = false;
     if (!SPARSE) {
@@ -542,9 +561,9 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
         fence_mbar_init();
         fence_proxy_async();
         // the queries start their way in at once: (d, row within the KV head's G*B rows, head); rows past the head read as zeros
-        mbar_arrive_expect_tx(bar(Q_FULL), n_mt * kTileBytes);
+        mbar_arrive_expect_tx(bar(Q_FULL), n_mt * (K8 ? kHalfBytes : kTileBytes));
         for (int mt = 0; mt < n_mt; ++mt)
-            for (int dh = 0; dh < 2; ++dh)
+            for (int dh = 0; dh < (K8 ? 1 : 2); ++dh)
                 for (int rb = 0; rb < 2; ++rb)
                     tma_load_3d(smem_u32(q_s + mt * kTileBytes + dh * kHalfBytes + rb * kBoxBytes), &maps.q, bar(Q_FULL), dh * 64,
                                 rg * 256 + mt * kTile + rb * 64, z);
@@ -605,10 +624,11 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                             for (int kh = 0; kh < 2; ++kh)
                                 if (paged_box_coords(kv, h, j_begin + i * kTile + kh * 64, pg_cur[kh], c1[kh], c2[kh], c3[kh], is_v ? nullptr : status)) bad |= 1 << kh;
                             if (!is_v) tile_bad_s[i & 7] = bad;     // ordered before K(i)'s FULL phase by the arrive below
-                            mbar_arrive_expect_tx(bar(FULL + slot), kTileBytes);
+                            const int n_dh = K8 && !is_v ? 1 : 2;
+                            mbar_arrive_expect_tx(bar(FULL + slot), n_dh * kHalfBytes);
                             const uint32_t dst = smem_u32(kv_s + slot * kTileBytes);
                             for (int kh = 0; kh < 2; ++kh)
-                                for (int dh = 0; dh < 2; ++dh)
+                                for (int dh = 0; dh < n_dh; ++dh)
                                     tma_load_4d_hint(dst + dh * kHalfBytes + kh * kBoxBytes, is_v ? &maps.v : &maps.k, bar(FULL + slot), dh * 64, c1[kh], c2[kh], c3[kh], is_v ? pol_v : pol_k);
                         }
                         if (is_v) {                            // tile i + 1 becomes current, tile i + 2 is looked up
@@ -629,17 +649,18 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                             issued = L + 1;
                             continue;
                         }
-                        mbar_arrive_expect_tx(bar(FULL + slot), kTileBytes);
+                        const int n_dh = K8 && !is_v ? 1 : 2;
+                        mbar_arrive_expect_tx(bar(FULL + slot), n_dh * kHalfBytes);
                         const uint32_t dst = smem_u32(kv_s + slot * kTileBytes);
                         for (int kh = 0; kh < 2; ++kh) {
                             if (!blk_chunk) {
                                 int c1, c2, c3;
                                 cache_box_coords(kv, p, h, j_begin + i * kTile + kh * 64, N, c1, c2, c3, nullptr);
-                                for (int dh = 0; dh < 2; ++dh)
+                                for (int dh = 0; dh < n_dh; ++dh)
                                     tma_load_4d_hint(dst + dh * kHalfBytes + kh * kBoxBytes, is_v ? &maps.v : &maps.k, bar(FULL + slot), dh * 64, c1, c2, c3, is_v ? pol_v : pol_k);
                             } else {
                                 const int row = (i == 0 && kh == 0) ? z * kv.B : blk_rows_total + 64;   // beyond the tensor: zero fill
-                                for (int dh = 0; dh < 2; ++dh)
+                                for (int dh = 0; dh < n_dh; ++dh)
                                     tma_load_2d(dst + dh * kHalfBytes + kh * kBoxBytes, is_v ? &maps.vb : &maps.kb, bar(FULL + slot), dh * 64, row);
                             }
                         }
@@ -668,7 +689,9 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     // Requests of a tile: (group of four consecutive list positions, d-half), 64 for a full tile, fewer for
                     // the last one; request o goes to warp o % 7, lane o / 7.  Each warp announces its share of the bytes.
                     const int pw = pt >> 5;
-                    const int n_req = ((i == n_tiles - 1 ? last_cols : kTile) >> 2) * 2;
+                    // (8-bit keys: a key row is one 128-byte piece, so a K tile takes half as many requests)
+                    const bool one_piece = K8 && !is_v;
+                    const int n_req = ((i == n_tiles - 1 ? last_cols : kTile) >> 2) * (one_piece ? 1 : 2);
                     const int mine = n_req > pw ? (n_req - pw + kSparseProducerWarps - 1) / kSparseProducerWarps : 0;
                     if (lane == 0) {
                         if (mine > 0) mbar_arrive_expect_tx(bar(FULL + slot), mine * 512);
@@ -677,7 +700,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     __syncwarp();
                     if (lane < mine) {
                         const int o = lane * kSparseProducerWarps + pw;
-                        const int r_in_tile = (o >> 1) * 4, dh = o & 1, t0 = i * kTile + r_in_tile;
+                        const int r_in_tile = (one_piece ? o : o >> 1) * 4, dh = one_piece ? 0 : o & 1, t0 = i * kTile + r_in_tile;
                         int rows[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
@@ -757,8 +780,8 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issue (one lane)
         if (lane == 0) {
-            const uint32_t idesc_qk = idesc_bf16_f32(kTile, false, false);   // S[128 rows][128 keys]
-            const uint32_t idesc_qk_last = idesc_bf16_f32(last_cols, false, false);
+            const uint32_t idesc_qk = K8 ? idesc_e4m3_f32(kTile) : idesc_bf16_f32(kTile, false, false);   // S[128 rows][128 keys]
+            const uint32_t idesc_qk_last = K8 ? idesc_e4m3_f32(last_cols) : idesc_bf16_f32(last_cols, false, false);
             const int nks_last = last_cols >> 4;                             // 16-key steps of the last tile's P V
             const uint32_t idesc_pv = idesc_bf16_f32(kD, false, true);       // O[128 rows][128 d], V is MN-major
             // The issuing thread runs in step with the tensor pipe (an MMA is accepted only as the previous one drains),
@@ -787,6 +810,11 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             auto qk = [&](int slot, int reg, int tile) {
                 const uint32_t a0 = q_lo + (tp ? 0u : (uint32_t)reg * kTileU), b0 = k_lo + (uint32_t)slot * kTileU;
                 const uint32_t idesc = SPARSE && tile == n_tiles - 1 ? idesc_qk_last : idesc_qk;
+                if (K8) {                                      // 32 one-byte elements of d per step, the row is one swizzle atom
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) umma_ss_f8(tmem_base + reg * 128, desc(a0 + ks * 2), desc(b0 + ks * 2), idesc, ks > 0);
+                    return;
+                }
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint32_t off = (ks >> 2) * kHalfU + (ks & 3) * 2;
