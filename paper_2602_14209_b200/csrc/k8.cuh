@@ -12,6 +12,7 @@
 // The codes of the cache are written once (and again for appended rows); queries and block keys are coded at every call.
 #pragma once
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace mage {
 namespace k8 {
@@ -91,6 +92,8 @@ __global__ void __launch_bounds__(256) block_code_kernel(KvView kv, const __nv_b
                                                          const float *__restrict__ k_scale, uint8_t *__restrict__ q8,
                                                          uint8_t *__restrict__ kb8, float *__restrict__ qk_scale) {
     __shared__ float red[8];
+    ptx::pdl_wait();                 // launched with programmatic serialization: nothing is read before the predecessor is done
+    ptx::pdl_launch_dependents();    // the pass that follows may set itself up meanwhile; it waits for this grid's end before reading
     const int z = blockIdx.x, p = z / kv.H_kv, h = z % kv.H_kv, tid = threadIdx.x;
     const size_t q_off = ((size_t)(p * kv.H_q + h * kv.G) * kv.B) * kD;
     const uint4 *qv = reinterpret_cast<const uint4 *>(q + q_off);

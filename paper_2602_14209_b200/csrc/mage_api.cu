@@ -193,7 +193,7 @@ static size_t k8_scratch_layout(const mage_kv_t *kv, size_t *off_kb8, size_t *of
 }
 // Codes of the call's queries and block keys (one small kernel in front of the pass that uses them).
 static mage_status launch_block_codes(const KvView &view, const K8 &k8, const __nv_bfloat16 *q, const __nv_bfloat16 *k_blk, cudaStream_t st) {
-    k8::block_code_kernel<<<view.P * view.H_kv, 256, 0, st>>>(view, q, k_blk, k8.k_scale, k8.q8, k8.kb8, k8.qk_scale);
+    launch_pdl(k8::block_code_kernel, dim3(view.P * view.H_kv), dim3(256), 0, st, view, q, k_blk, k8.k_scale, k8.q8, k8.kb8, k8.qk_scale);
     return launch_check();
 }
 

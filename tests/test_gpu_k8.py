@@ -57,40 +57,43 @@ def _run(batch, w, paged, k, steps=(0, 1)):
             "keff": keff.cpu().numpy(), "out_sp": out_sp.float().cpu().numpy(), "k_scale": k8.k_scale.cpu().numpy()}
 
 
-def _check(o, batch, w, res, k, steps=(0, 1)):
+def _check(o, batch, w, res, k, steps=(0, 1), pairs=None):
+    """Compare with the oracle, head by head; pairs = [(problem, KV head), ...] restricts the comparison (default: all)."""
     f = lambda t: t.float().cpu().numpy()
+    G = w.G
     diag = {"o_max": 0.0, "score_rel": 0.0, "swaps": 0, "sp_max": 0.0}
     for p, n in enumerate(batch["seq_lens"].tolist()):
-        Kc, Vc = f(batch["kc"][p, :, :n]), f(batch["vc"][p, :, :n])
-        Q0, Kb0, Vb0 = f(batch["q"][steps[0], p]), f(batch["kb"][steps[0], p]), f(batch["vb"][steps[0], p])
-        Qc, Kcc, Kbc, s_q, s_k = o.k8_quantize_block(Q0, Kc, Kb0)
-        # the cache's codes and scales are the oracle's, bit for bit
-        assert np.array_equal(res["k_scale"][p], s_k)
-        for h in range(w.H_kv):
-            got = _codes_of(res["k8"], res["kv"], res["table"], p, h, n)
-            assert np.array_equal(got, Kcc[h]) and np.array_equal(np.signbit(got), np.signbit(Kcc[h]))
-        O = o.k8_exact_block_attn(Qc, Kcc, Vc, Kbc, Vb0, s_q, s_k)
-        err = np.abs(res["out"][p] - O)
-        assert np.isfinite(res["out"][p]).all() and err.max() <= H.O_MAX_ABS and err.mean() <= H.O_MEAN_ABS, (p, err.max(), err.mean())
-        diag["o_max"] = max(diag["o_max"], err.max())
+        heads = [h for h in range(w.H_kv) if pairs is None or (p, h) in pairs]
         assert res["keff"][p] == min(k, n)
-        if n > 0:
-            sc = o.k8_block_score(Qc, Kcc, s_q, s_k)
-            rel = np.max(np.abs(res["scores"][p, :, :n] - sc) / sc)
-            assert rel <= H.SCORE_REL, (p, rel)
-            diag["score_rel"] = max(diag["score_rel"], rel)
-            assert (res["scores"][p, :, n:] == -1.0).all()
-            for h in range(w.H_kv):
-                diag["swaps"] += H.check_topk_band(sc[h], res["idx"][p, h], k, n)
-        else:
+        if n == 0:
             assert (res["idx"][p] == -1).all()
-        # reuse step: its own queries and block keys are coded at the call; the cache codes are the same
-        Q1, Kb1, Vb1 = f(batch["q"][steps[1], p]), f(batch["kb"][steps[1], p]), f(batch["vb"][steps[1], p])
-        Qc1, _, Kbc1, s_q1, _ = o.k8_quantize_block(Q1, Kc, Kb1)
-        Os = o.k8_sparse_block_attn(Qc1, Kcc, Vc, Kbc1, Vb1, res["idx"][p], int(res["keff"][p]), s_q1, s_k)
-        e = np.abs(res["out_sp"][p] - Os)
-        assert np.isfinite(res["out_sp"][p]).all() and e.max() <= H.O_MAX_ABS and e.mean() <= H.O_MEAN_ABS, (p, e.max(), e.mean())
-        diag["sp_max"] = max(diag["sp_max"], e.max())
+        for h in heads:
+            g = slice(h * G, (h + 1) * G)
+            Kc, Vc = f(batch["kc"][p, h:h + 1, :n]), f(batch["vc"][p, h:h + 1, :n])
+            Q0, Kb0, Vb0 = f(batch["q"][steps[0], p, g]), f(batch["kb"][steps[0], p, h:h + 1]), f(batch["vb"][steps[0], p, h:h + 1])
+            Qc, Kcc, Kbc, s_q, s_k = o.k8_quantize_block(Q0, Kc, Kb0)
+            # the cache's codes and scales are the oracle's, bit for bit
+            assert res["k_scale"][p, h] == s_k[0]
+            got = _codes_of(res["k8"], res["kv"], res["table"], p, h, n)
+            assert np.array_equal(got, Kcc[0]) and np.array_equal(np.signbit(got), np.signbit(Kcc[0]))
+            O = o.k8_exact_block_attn(Qc, Kcc, Vc, Kbc, Vb0, s_q, s_k)
+            err = np.abs(res["out"][p, g] - O)
+            assert np.isfinite(res["out"][p, g]).all() and err.max() <= H.O_MAX_ABS and err.mean() <= H.O_MEAN_ABS, (p, h, err.max(), err.mean())
+            diag["o_max"] = max(diag["o_max"], err.max())
+            if n > 0:
+                sc = o.k8_block_score(Qc, Kcc, s_q, s_k)[0]
+                rel = np.max(np.abs(res["scores"][p, h, :n] - sc) / sc)
+                assert rel <= H.SCORE_REL, (p, h, rel)
+                diag["score_rel"] = max(diag["score_rel"], rel)
+                assert (res["scores"][p, h, n:] == -1.0).all()
+                diag["swaps"] += H.check_topk_band(sc, res["idx"][p, h], k, n)
+            # reuse step: its own queries and block keys are coded at the call; the cache codes are the same
+            Q1, Kb1, Vb1 = f(batch["q"][steps[1], p, g]), f(batch["kb"][steps[1], p, h:h + 1]), f(batch["vb"][steps[1], p, h:h + 1])
+            Qc1, _, Kbc1, s_q1, _ = o.k8_quantize_block(Q1, Kc, Kb1)
+            Os = o.k8_sparse_block_attn(Qc1, Kcc, Vc, Kbc1, Vb1, res["idx"][p, h:h + 1], int(res["keff"][p]), s_q1, s_k)
+            e = np.abs(res["out_sp"][p, g] - Os)
+            assert np.isfinite(res["out_sp"][p, g]).all() and e.max() <= H.O_MAX_ABS and e.mean() <= H.O_MEAN_ABS, (p, h, e.max(), e.mean())
+            diag["sp_max"] = max(diag["sp_max"], e.max())
     return diag
 
 
@@ -112,6 +115,37 @@ def test_k8_block_against_oracle(oracle_mod, case, paged):
     res = _run(batch, w, paged, k)
     diag = _check(oracle_mod, batch, w, res, k)
     print(name, "paged" if paged else "contiguous", diag)
+
+
+def _global_properties(batch, res, k):
+    """What holds at any size: finite outputs, score rows that sum to one, index rows ascending, in range, -1 padded."""
+    assert np.isfinite(res["out"]).all() and np.isfinite(res["out_sp"]).all()
+    for p, n in enumerate(batch["seq_lens"].tolist()):
+        k_eff = min(k, n)
+        assert res["keff"][p] == k_eff
+        np.testing.assert_allclose(res["scores"][p, :, :n].astype(np.float64).sum(axis=1), 1.0, rtol=2e-5)
+        idx = res["idx"][p, :, :k_eff]
+        assert (idx >= 0).all() and (idx < n).all() and (np.diff(idx, axis=1) > 0).all() and (res["idx"][p, :, k_eff:] == -1).all()
+
+
+def test_k8_cfg2_qwen_32k_every_head(oracle_mod):
+    w = W.CONFIGS["cfg2_qwen_32k"]
+    batch = W.make_batch(w, device="cuda", steps=2)
+    res = _run(batch, w, False, w.k)
+    _global_properties(batch, res, w.k)
+    print("cfg2 k8", _check(oracle_mod, batch, w, res, w.k))
+    # the planted heavy positions still dominate the selection made from 8-bit keys and queries
+    for h in range(w.H_kv):
+        assert len(set(res["idx"][0, h].tolist()) & set(batch["heavy"][0][h].tolist())) > 0.5 * w.k
+
+
+def test_k8_cfg3_qwen_128k_28_layers_sampled(oracle_mod):
+    """The benchmark workload in its batched launch: properties everywhere, four (layer, head) pairs element by element."""
+    w = W.CONFIGS["cfg3_qwen_128k_x28"]
+    batch = W.make_batch(w, device="cuda", steps=2)
+    res = _run(batch, w, False, w.k)
+    _global_properties(batch, res, w.k)
+    print("cfg3 k8", _check(oracle_mod, batch, w, res, w.k, pairs=[(0, 0), (9, 1), (18, 2), (27, 3)]))
 
 
 def test_k8_block_keys_clamp_at_the_cache_scale(oracle_mod):
