@@ -444,6 +444,33 @@ def main():
             stages["quest_step_ms_cold_l2"] = stages["quest_select_ms_cold_l2"] + timed(qsp, True, 5)
             stages["quest_summary_bytes"] = 2 * pmin.numel() * 2
             del pmin, pmax, psc
+        # Step 1 and the reuse step with the keys (and queries) in 8 bits, beside the 16-bit calls, alternating so that both see
+        # the same clocks; agreement of the two selections (|S_8 & S_16| / k, mean over heads).  Not part of the headline.
+        try:
+            k8 = mb.K8Keys(kv)
+            stages["k8_quantize_cache_ms"] = timed(lambda: k8.quantize(0, ba.status), False, 3)
+            s16 = lambda: mb.mage_exact_select(kv, q_d[0], kb_d[0], vb_d[0], ba.sm_scale, outs[0], ba.scores, ba.workspace, ba.status)
+            s8 = lambda: mb.mage_exact_select_k8(kv, k8, q_d[0], kb_d[0], vb_d[0], ba.sm_scale, outs[0], ba.scores, ba.workspace, ba.status)
+            t16, t8 = [], []
+            for _ in range(5):
+                t16.append(timed(s16, False, 1)); t8.append(timed(s8, False, 1))
+            stages["exact_select_ms_alternating"], stages["k8_exact_select_ms_alternating"] = sorted(t16)[2], sorted(t8)[2]
+            s16(); tk(); torch.cuda.synchronize()
+            idx16 = ba.indices.clone()
+            s8(); tk(); torch.cuda.synchronize()
+            same = 0
+            for p_ in range(kv.P):
+                for h_ in range(kv.H_kv):
+                    same += len(set(idx16[p_, h_].tolist()) & set(ba.indices[p_, h_].tolist()) - {-1})
+            stages["k8_selection_overlap_with_16bit"] = same / max(1, int(ba.k_eff.sum().item()) * kv.H_kv)
+            sp8 = lambda: mb.mage_sparse_block_attn_k8(kv, k8, q_d[1], kb_d[1], vb_d[1], ba.indices, ba.k_eff, w.k, ba.sm_scale, outs[1], ba.workspace, ba.status)
+            sp8(); torch.cuda.synchronize()
+            stages["k8_sparse_step_ms_cold_l2"] = timed(sp8, True)
+            stages["k8_key_bytes_per_token_head"] = 128
+            del k8
+            s16(); tk(); torch.cuda.synchronize()          # leave the 16-bit selection in place for what follows
+        except mb.MageError as e:                          # a description the 8-bit calls do not take
+            stages["k8_unavailable"] = str(e)
         del flush
         # The same block issued layer by layer, as a model would (config 3 "timed back-to-back"): one exact_select, one
         # top-k (select stream) and T-1 sparse launches per layer; plain launches, and replayed from a CUDA graph.

@@ -97,9 +97,25 @@ __global__ void __launch_bounds__(256) block_code_kernel(KvView kv, const __nv_b
     const int z = blockIdx.x, p = z / kv.H_kv, h = z % kv.H_kv, tid = threadIdx.x;
     const size_t q_off = ((size_t)(p * kv.H_q + h * kv.G) * kv.B) * kD;
     const uint4 *qv = reinterpret_cast<const uint4 *>(q + q_off);
-    const int n_q8 = kv.M * (kD / 8);                            // 8-element pieces of the head's queries
+    const int n_q16 = kv.M * (kD / 16);                          // 16-element pieces of the head's queries
+    // up to 256 rows stay in registers between the two passes (eight pieces per thread); longer heads are read again
+    uint4 keep[16];
     float m = 0.f;
-    for (int i = tid; i < n_q8; i += 256) m = amax8(qv[i], m);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const int j = tid + u * 256;
+        if (j < n_q16) {
+            keep[2 * u] = qv[2 * j];
+            keep[2 * u + 1] = qv[2 * j + 1];
+            m = amax8(keep[2 * u + 1], amax8(keep[2 * u], m));
+        }
+    }
+    for (int j = tid + 2048; j < n_q16; j += 256) m = amax8(qv[2 * j + 1], amax8(qv[2 * j], m));
+    const uint4 *bv = reinterpret_cast<const uint4 *>(k_blk + (size_t)z * kv.B * kD);
+    uint4 kb0 = make_uint4(0, 0, 0, 0), kb1 = kb0, kb2 = kb0, kb3 = kb0;      // the block's keys: B <= 64 rows, two pieces per thread
+    const int n_b16 = kv.B * (kD / 16);
+    if (tid < n_b16) { kb0 = bv[2 * tid]; kb1 = bv[2 * tid + 1]; }
+    if (tid + 256 < n_b16) { kb2 = bv[2 * (tid + 256)]; kb3 = bv[2 * (tid + 256) + 1]; }
 #pragma unroll
     for (int w = 16; w; w >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, w));
     if ((tid & 31) == 0) red[tid >> 5] = m;
@@ -109,12 +125,16 @@ __global__ void __launch_bounds__(256) block_code_kernel(KvView kv, const __nv_b
     for (int w = 1; w < 8; ++w) m = fmaxf(m, red[w]);
     const float s_q = scale_of(m), s_k = k_scale[z];
     if (tid == 0) qk_scale[z] = s_q * s_k;
-    for (int i = tid; i < kv.M * (kD / 16); i += 256)
-        *reinterpret_cast<uint4 *>(q8 + q_off + (size_t)i * 16) = code16(qv[2 * i], qv[2 * i + 1], s_q);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const int j = tid + u * 256;
+        if (j < n_q16) *reinterpret_cast<uint4 *>(q8 + q_off + (size_t)j * 16) = code16(keep[2 * u], keep[2 * u + 1], s_q);
+    }
+    for (int j = tid + 2048; j < n_q16; j += 256)
+        *reinterpret_cast<uint4 *>(q8 + q_off + (size_t)j * 16) = code16(qv[2 * j], qv[2 * j + 1], s_q);
     const size_t b_off = (size_t)z * kv.B * kD;
-    const uint4 *bv = reinterpret_cast<const uint4 *>(k_blk + b_off);
-    for (int i = tid; i < kv.B * (kD / 16); i += 256)
-        *reinterpret_cast<uint4 *>(kb8 + b_off + (size_t)i * 16) = code16(bv[2 * i], bv[2 * i + 1], s_k);
+    if (tid < n_b16) *reinterpret_cast<uint4 *>(kb8 + b_off + (size_t)tid * 16) = code16(kb0, kb1, s_k);
+    if (tid + 256 < n_b16) *reinterpret_cast<uint4 *>(kb8 + b_off + (size_t)(tid + 256) * 16) = code16(kb2, kb3, s_k);
 }
 
 }  // namespace k8
