@@ -93,7 +93,7 @@ class ClockSampler(threading.Thread):
                 "samples": len(self.samples), "power_w_max": max(x[2] for x in self.samples), "source": "nvml"}
 
 
-def stage_bytes_flops(w, lens):
+def stage_bytes_flops(w, lens, key_bytes=2):
     """Algorithmic traffic and work of each stage for one block (all problems).
 
     Stage 1 must read every cached K and V row once (512 B per cached token per KV head), Q and the block's K/V,
@@ -105,21 +105,22 @@ def stage_bytes_flops(w, lens):
     tok = sum(lens)
     qo = len(lens) * w.H_q * w.B * d * 2
     kvb = len(lens) * w.H_kv * w.B * d * 2 * 2
-    s1_bytes = tok * w.H_kv * (2 * d * 2 + 4) + 2 * qo + kvb
-    s1_attn_bytes = tok * w.H_kv * 2 * d * 2 + qo + kvb            # the attention kernel alone
+    row = d * key_bytes + d * 2                                     # one cached token of one KV head: its key and its value
+    s1_bytes = tok * w.H_kv * (row + 4) + 2 * qo + kvb
+    s1_attn_bytes = tok * w.H_kv * row + qo + kvb                   # the attention kernel alone
     s1_flops_attn = sum(4 * M * (n + w.B) * d * w.H_kv for n in lens)
     s1_flops_score = sum(2 * M * n * d * w.H_kv for n in lens)
     keff = [min(w.k, n) for n in lens]
-    s3_bytes = sum(ke * w.H_kv * (2 * d * 2 + 4) for ke in keff) + 2 * qo + kvb
+    s3_bytes = sum(ke * w.H_kv * (row + 4) for ke in keff) + 2 * qo + kvb
     s3_flops = sum(4 * M * (ke + w.B) * d * w.H_kv for ke in keff)
     return {"s1_bytes": s1_bytes, "s1_attn_bytes": s1_attn_bytes, "s1_flops_attn": s1_flops_attn,
             "s1_flops_score": s1_flops_score, "s3_bytes": s3_bytes, "s3_flops": s3_flops}
 
 
-def config_of(w, lens, world, kernels, parallelism=None):
+def config_of(w, lens, world, kernels, parallelism=None, key_bytes=2):
     """The `config` object of the JSON line; both arms print the same keys."""
     return {"workload": w.name, "H_q": w.H_q, "H_kv": w.H_kv, "d": w.d, "N": w.N, "B": w.B, "k": w.k, "T": w.T,
-            "problems": w.P, "cached_tokens": sum(lens), "kv_bytes": sum(lens) * w.H_kv * 512,
+            "problems": w.P, "cached_tokens": sum(lens), "kv_bytes": sum(lens) * w.H_kv * (w.d * key_bytes + w.d * 2),
             "l2_policy": "inputs_larger_than_l2 (KV cache streamed every step evicts L2)",
             "parallelism": parallelism or f"replicas x{world} (independent blocks, no collective)", "kernels": kernels}
 
@@ -218,6 +219,9 @@ def main():
     ap.add_argument("--shard", default="replicas", choices=["replicas", "kv_head"],
                     help="N > 1: replicas = every rank runs its own block (weak scaling); kv_head = the ranks split the KV heads of ONE "
                          "block between them, no collective on the data path (strong scaling)")
+    ap.add_argument("--keys", default="bf16", choices=["bf16", "e4m3"],
+                    help="e4m3: the variant with keys and queries as 8-bit codes (values bf16), timed the same way; no stage breakdown, "
+                         "no CPU leg; the default line and every number quoted for the metric are bf16")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-stage-breakdown", action="store_true")
     ap.add_argument("--bootstrap-only", action="store_true", help="start the ranks, reduce a stand-in time over them and exit (no kernels)")
@@ -281,13 +285,19 @@ def main():
         kv = mb.KVCache(k_pool, v_pool, w.H_q, w.B, seq_lens=batch["seq_lens"], block_table=table, N_max=batch["N_max"], flags=flags)
     else:
         kv = mb.KVCache(batch["kc"], batch["vc"], w.H_q, w.B, seq_lens=batch["seq_lens"], flags=flags)
-    ba = BlockAttention(kv, w.k)
+    k8_keys = None
+    if args.keys == "e4m3":
+        if args.simt or kv_head_sharded:
+            raise SystemExit("--keys e4m3 runs on the tensor-core kernels, unsharded")
+        k8_keys = mb.K8Keys(kv).quantize()              # one-off coding of the cache, outside the timed regions
+        args.no_stage_breakdown = args.no_cpu_baseline = True
+    ba = BlockAttention(kv, w.k, k8=k8_keys)
     T = w.T
     q_d = [batch["q"][t] for t in range(T)]
     kb_d = [batch["kb"][t] for t in range(T)]
     vb_d = [batch["vb"][t] for t in range(T)]
     outs = [torch.empty_like(ba.out) for _ in range(T)]
-    sf = stage_bytes_flops(w, lens)
+    sf = stage_bytes_flops(w, lens, key_bytes=1 if k8_keys is not None else 2)
     main_stream = torch.cuda.current_stream()
 
     def barrier():
@@ -560,11 +570,16 @@ def main():
         roofline["frac"] = roofline["achieved"] / roofline["peak"]
     else:
         achieved = sf["s1_flops_attn"] / attn_avg_ms / 1e9
-        roofline = {"bound": "tensor", "kernel": "tc::attn_kernel<false> (Step-1 exact pass over prefix + block keys)", "achieved": achieved,
-                    "peak": peaks["bf16_tflops"] if burst_regime else peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+        # 8-bit keys: half of the kernel's flops (Q K^T) run on the e4m3 path, whose peak is the measured bf16 peak times the
+        # nominal ratio 2, the other half (P V) on bf16: the blended peak is total / (1/2 / 2P + 1/2 / P) = 4/3 P
+        blend = 4.0 / 3.0 if k8_keys is not None else 1.0
+        roofline = {"bound": "tensor", "kernel": "tc::attn_kernel<false> (Step-1 exact pass over prefix + block keys)"
+                                                 + (", Q K^T in e4m3, P V in bf16" if k8_keys is not None else ""), "achieved": achieved,
+                    "peak": blend * (peaks["bf16_tflops"] if burst_regime else peaks["bf16_tflops_sustained"]), "unit": "TFLOP/s",
                     "peak_source": f"bf16 cuBLAS {'burst' if burst_regime else 'sustained'}, {peaks['source']}: "
-                                   + ("median SM clock >= 0.95 max and no sw_power_cap sample" if burst_regime else "sw_power_cap sampled or SM clock below 0.95 max"),
-                    "frac_burst": achieved / peaks["bf16_tflops"], "frac_sustained": achieved / peaks["bf16_tflops_sustained"],
+                                   + ("median SM clock >= 0.95 max and no sw_power_cap sample" if burst_regime else "sw_power_cap sampled or SM clock below 0.95 max")
+                                   + ("; x 4/3: half of the flops at the nominal 2x e4m3 rate" if k8_keys is not None else ""),
+                    "frac_burst": achieved / (blend * peaks["bf16_tflops"]), "frac_sustained": achieved / (blend * peaks["bf16_tflops_sustained"]),
                     "issued_over_useful_flops": float(-(-w.M // 128) * 128) / w.M, "traffic": None}
         roofline["frac"] = roofline["achieved"] / roofline["peak"]
     roofline["hbm_view"] = {"achieved_gbs": sf["s1_attn_bytes"] / attn_avg_ms / 1e6, "peak_gbs": peaks["hbm_gbs"],
@@ -574,13 +589,15 @@ def main():
     if os.path.exists(prof):
         for ln in open(prof):
             f = ln.split(None, 3)
-            if len(f) >= 3 and not ln.startswith("#") and f[0] == ("simt" if args.simt else "default") and f[1] == w.name:
+            if len(f) >= 3 and not ln.startswith("#") and f[0] == ("simt" if args.simt else "default") and f[1] == w.name and k8_keys is None:
                 roofline["traffic"] = int(f[2])
                 roofline["traffic_source"] = f[3].strip() if len(f) > 3 else "ncu capture, see profiles/traffic.txt"
     # the stages the benchmark spec names, each against the roof that binds it
     s1_ms_all = (sum(attn_ms) + sum(comb_ms) + sum(score_ms)) / len(attn_ms)
     s1_flops = sf["s1_flops_attn"] + sf["s1_flops_score"]
     tensor_peak = peaks["bf16_tflops"] if burst_regime else peaks["bf16_tflops_sustained"]
+    if k8_keys is not None:      # Step 1 as a whole: two of its three contractions (both Q K^T) on the e4m3 path: 1 / (2/3 / 2 + 1/3) = 3/2
+        tensor_peak *= 1.5
     roofline_stages = {
         "step1_exact_select": {"bound": "tensor", "achieved": s1_flops / s1_ms_all / 1e9, "peak": tensor_peak, "unit": "TFLOP/s",
                                "frac": s1_flops / s1_ms_all / 1e9 / tensor_peak, "flops": s1_flops, "ms": s1_ms_all,
@@ -606,9 +623,9 @@ def main():
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "strong" if kv_head_sharded else "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
-        "config": config_of(w_full, lens, world, "simt" if args.simt else "default",
-                            f"kv_head x{world} (each rank owns H_kv/{world} KV heads of every layer; no collective)" if kv_head_sharded else None),
+        "dtype": "bf16" if k8_keys is None else "e4m3 (Q K^T) + bf16 (P V)", "data": "synthetic",
+        "config": config_of(w_full, lens, world, "simt" if args.simt else ("default" if k8_keys is None else "default, keys and queries e4m3"),
+                            f"kv_head x{world} (each rank owns H_kv/{world} KV heads of every layer; no collective)" if kv_head_sharded else None, key_bytes=1 if k8_keys is not None else 2),
         "clocks": clocks, "gpu_launches": launches, "dev_status": status,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "roofline": roofline, "roofline_stages": roofline_stages, "cpu_baseline": cpu_baseline, "stages": stages,

@@ -331,6 +331,11 @@ mage_status mage_k8_quantize_cache(const mage_kv_t *kv, int32_t row_begin, void 
 mage_status mage_exact_select_k8(const mage_kv_t *kv, const mage_k8_t *k8, const void *q, const void *k_blk, const void *v_blk,
                                  float sm_scale, void *out, float *scores, void *workspace, size_t workspace_bytes,
                                  uint32_t *dev_status, void *stream);
+/* The same call with four caller events recorded between its kernels, as mage_exact_select_events (the block-code kernel
+ * falls between events[0] and events[1], with the exact pass). */
+mage_status mage_exact_select_k8_events(const mage_kv_t *kv, const mage_k8_t *k8, const void *q, const void *k_blk, const void *v_blk,
+                                        float sm_scale, void *out, float *scores, void *workspace, size_t workspace_bytes,
+                                        uint32_t *dev_status, void *stream, void **events);
 mage_status mage_sparse_block_attn_k8(const mage_kv_t *kv, const mage_k8_t *k8, const void *q, const void *k_blk, const void *v_blk,
                                       const int32_t *indices, const int32_t *k_eff, int32_t k, float sm_scale, void *out,
                                       void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream);

@@ -44,7 +44,7 @@ class mage_kv_t(ctypes.Structure):
 
 
 EXPORTS = ("mage_pruned_workspace_bytes", "mage_exact_select_pruned", "mage_quest_workspace_bytes", "mage_quest_build", "mage_quest_select", "mage_append_block", "mage_workspace_bytes", "mage_exact_select", "mage_exact_select_events", "mage_exact_select_static", "mage_exact_attn", "mage_select_scores", "mage_topk", "mage_sparse_block_attn",
-           "mage_k8_scratch_bytes", "mage_k8_quantize_cache", "mage_exact_select_k8", "mage_sparse_block_attn_k8",
+           "mage_k8_scratch_bytes", "mage_k8_quantize_cache", "mage_exact_select_k8", "mage_exact_select_k8_events", "mage_sparse_block_attn_k8",
            "mage_status_string", "mage_launch_count")
 
 
@@ -93,6 +93,8 @@ def load():
     lib.mage_exact_select_k8.restype = ctypes.c_int
     lib.mage_exact_select_k8.argtypes = [ctypes.POINTER(mage_kv_t), ctypes.POINTER(mage_k8_t), vp, vp, vp, ctypes.c_float, vp, vp, vp,
                                          ctypes.c_size_t, vp, vp]
+    lib.mage_exact_select_k8_events.restype = ctypes.c_int
+    lib.mage_exact_select_k8_events.argtypes = lib.mage_exact_select_k8.argtypes + [ctypes.POINTER(ctypes.c_void_p)]
     lib.mage_sparse_block_attn_k8.restype = ctypes.c_int
     lib.mage_sparse_block_attn_k8.argtypes = [ctypes.POINTER(mage_kv_t), ctypes.POINTER(mage_k8_t), vp, vp, vp, vp, vp, i32, ctypes.c_float,
                                               vp, vp, ctypes.c_size_t, vp, vp]
@@ -264,11 +266,19 @@ class K8Keys:
         return self
 
 
-def mage_exact_select_k8(kv: KVCache, k8: K8Keys, q, k_blk, v_blk, sm_scale: float, out, scores, workspace, dev_status=None, stream=None):
-    """mage_exact_select with the keys (and queries) in 8 bits (see mage.h)."""
-    rc = load().mage_exact_select_k8(ctypes.byref(kv.c), ctypes.byref(k8.c), _ptr(q), _ptr(k_blk), _ptr(v_blk), float(sm_scale), _ptr(out),
-                                     _ptr(scores), _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(dev_status),
-                                     _stream(stream))
+def mage_exact_select_k8(kv: KVCache, k8: K8Keys, q, k_blk, v_blk, sm_scale: float, out, scores, workspace, dev_status=None, stream=None,
+                         events=None):
+    """mage_exact_select with the keys (and queries) in 8 bits (see mage.h); ``events`` as in ``mage_exact_select``."""
+    args = (ctypes.byref(kv.c), ctypes.byref(k8.c), _ptr(q), _ptr(k_blk), _ptr(v_blk), float(sm_scale), _ptr(out), _ptr(scores),
+            _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream(stream))
+    if events is None:
+        rc = load().mage_exact_select_k8(*args)
+    else:
+        for e in events:
+            if not e.cuda_event:
+                e.record()
+        handles = (ctypes.c_void_p * 4)(*[ctypes.c_void_p(e.cuda_event) for e in events])
+        rc = load().mage_exact_select_k8_events(*args, handles)
     if rc != MAGE_OK:
         raise MageError(rc, "mage_exact_select_k8")
 

@@ -500,9 +500,9 @@ mage_status mage_k8_quantize_cache(const mage_kv_t *kv, int32_t row_begin, void 
     return MAGE_OK;
 }
 
-mage_status mage_exact_select_k8(const mage_kv_t *kv, const mage_k8_t *k8, const void *q, const void *k_blk, const void *v_blk,
-                                 float sm_scale, void *out, float *scores, void *workspace, size_t workspace_bytes,
-                                 uint32_t *dev_status, void *stream) {
+mage_status mage_exact_select_k8_events(const mage_kv_t *kv, const mage_k8_t *k8, const void *q, const void *k_blk, const void *v_blk,
+                                        float sm_scale, void *out, float *scores, void *workspace, size_t workspace_bytes,
+                                        uint32_t *dev_status, void *stream, void **events) {
     if (!kv || !k8) return MAGE_ERR_INVALID_ARG;
     mage_kv_t kvc = *kv;
     kvc.k_cache = k8->k8_cache;                            // the 16-bit keys are not read
@@ -518,7 +518,14 @@ mage_status mage_exact_select_k8(const mage_kv_t *kv, const mage_k8_t *k8, const
     const KvView view = make_view(&kvc);
     return launch_exact_select(&kvc, view, plan, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_blk),
                                static_cast<const __nv_bfloat16 *>(v_blk), sm_scale, static_cast<__nv_bfloat16 *>(out), scores,
-                               static_cast<float *>(workspace), dev_status, static_cast<cudaStream_t>(stream), nullptr, false, nullptr, 0, &a);
+                               static_cast<float *>(workspace), dev_status, static_cast<cudaStream_t>(stream),
+                               reinterpret_cast<cudaEvent_t *>(events), false, nullptr, 0, &a);
+}
+
+mage_status mage_exact_select_k8(const mage_kv_t *kv, const mage_k8_t *k8, const void *q, const void *k_blk, const void *v_blk,
+                                 float sm_scale, void *out, float *scores, void *workspace, size_t workspace_bytes,
+                                 uint32_t *dev_status, void *stream) {
+    return mage_exact_select_k8_events(kv, k8, q, k_blk, v_blk, sm_scale, out, scores, workspace, workspace_bytes, dev_status, stream, nullptr);
 }
 
 mage_status mage_sparse_block_attn_k8(const mage_kv_t *kv, const mage_k8_t *k8, const void *q, const void *k_blk, const void *v_blk,

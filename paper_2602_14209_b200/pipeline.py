@@ -18,10 +18,11 @@ class BlockAttention:
     """Owns the outputs and scratch of one batch of problems and issues the three library calls."""
 
     def __init__(self, kv: mb.KVCache, k: int, sm_scale: Optional[float] = None, select_stream: Optional[torch.cuda.Stream] = None,
-                 buffers: Optional[dict] = None):
+                 buffers: Optional[dict] = None, k8: Optional[mb.K8Keys] = None):
         """``buffers`` lets several instances (e.g. one per layer) live in slices of shared tensors: keys out, scores,
-        indices, k_eff, status, workspace; anything missing is allocated here."""
-        self.kv, self.k = kv, int(k)
+        indices, k_eff, status, workspace; anything missing is allocated here.  ``k8``: the cache's keys as 8-bit codes
+        (already quantised); Step 1 and the reuse steps then go through the ``*_k8`` calls."""
+        self.kv, self.k, self.k8 = kv, int(k), k8
         self.sm_scale = float(kv.d) ** -0.5 if sm_scale is None else float(sm_scale)
         dev = kv.device
         b = buffers or {}
@@ -38,6 +39,10 @@ class BlockAttention:
     def exact_select(self, q, k_blk, v_blk, out=None, stream=None, events=None):
         """Step 1 on ``stream`` (default: current): exact attention -> out, block scores -> self.scores."""
         out = self.out if out is None else out
+        if self.k8 is not None:
+            mb.mage_exact_select_k8(self.kv, self.k8, q, k_blk, v_blk, self.sm_scale, out, self.scores, self.workspace, self.status,
+                                    stream, events)
+            return out
         mb.mage_exact_select(self.kv, q, k_blk, v_blk, self.sm_scale, out, self.scores, self.workspace, self.status, stream,
                              events)
         return out
@@ -45,6 +50,8 @@ class BlockAttention:
     def exact_attn(self, q, k_blk, v_blk, out=None, stream=None):
         """Step 1's attention alone on ``stream`` (default: current); pair it with ``select_scores_async``."""
         out = self.out if out is None else out
+        if self.k8 is not None:
+            raise NotImplementedError("the two halves of Step 1 on their own exist for 16-bit keys only")
         mb.mage_exact_attn(self.kv, q, k_blk, v_blk, self.sm_scale, out, self.workspace, self.status, stream)
         return out
 
@@ -59,6 +66,8 @@ class BlockAttention:
         """The paper's two-stream Phase 1: block scores and top-k on the select stream from the queries alone, beside
         whatever the main stream does (its attention, then the FFN).  Uses a workspace of its own (allocated on first use),
         since the main stream's Step 1 may be using ``self.workspace`` at the same time.  Follow with ``join()``."""
+        if self.k8 is not None:
+            raise NotImplementedError("the two halves of Step 1 on their own exist for 16-bit keys only")
         main = torch.cuda.current_stream() if main_stream is None else main_stream
         if workspace is None:
             workspace = self.select_workspace()
@@ -86,6 +95,10 @@ class BlockAttention:
     def sparse_step(self, q, k_blk, v_blk, out=None, stream=None):
         """One reuse step (Phase 2) with the index sets fixed at Step 1."""
         out = self.out if out is None else out
+        if self.k8 is not None:
+            mb.mage_sparse_block_attn_k8(self.kv, self.k8, q, k_blk, v_blk, self.indices, self.k_eff, self.k, self.sm_scale, out,
+                                         self.workspace, self.status, stream)
+            return out
         mb.mage_sparse_block_attn(self.kv, q, k_blk, v_blk, self.indices, self.k_eff, self.k, self.sm_scale, out,
                                   self.workspace, self.status, stream)
         return out
