@@ -211,3 +211,74 @@ def test_k8_refusals():
         mb.mage_exact_select_k8(kv2, bad, batch["q"][0], batch["kb"][0], batch["vb"][0], kv.d ** -0.5, out, scores, kv2.new_workspace(64))
     assert e.value.code == -1
     torch.cuda.synchronize()
+
+
+def test_k8_through_block_attention_matches_the_direct_calls():
+    """pipeline.BlockAttention(k8=...) issues the same calls (Step 1 with events, top-k on the select stream, reuse steps)."""
+    from paper_2602_14209_b200.pipeline import BlockAttention
+    w = W.Workload("pipe", H_q=14, H_kv=2, N=1200, B=32, k=256, T=3, P=2, n_heavy=64, ragged_min=500, seed=16)
+    batch = W.make_batch(w, device="cuda", steps=3)
+    res = _run(batch, w, False, w.k)                                   # direct calls: Step 1 on step 0, reuse step on step 1
+    kv = res["kv"]
+    ba = BlockAttention(kv, w.k, k8=res["k8"])
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    outs = ba.run_block([batch["q"][t] for t in range(3)], [batch["kb"][t] for t in range(3)], [batch["vb"][t] for t in range(3)], events=ev)
+    torch.cuda.synchronize()
+    assert int(ba.status.item()) == 0
+    assert np.array_equal(ba.indices.cpu().numpy(), res["idx"]) and np.array_equal(ba.k_eff.cpu().numpy(), res["keff"])
+    n = batch["seq_lens"].tolist()
+    for p in range(w.P):
+        assert np.array_equal(ba.scores[p, :, :n[p]].cpu().numpy(), res["scores"][p, :, :n[p]])
+    assert ev[0].elapsed_time(ev[3]) > 0
+    outs2 = [torch.empty_like(ba.out) for _ in range(3)]
+    ba.run_block([batch["q"][t] for t in range(3)], [batch["kb"][t] for t in range(3)], [batch["vb"][t] for t in range(3)], outs2)
+    torch.cuda.synchronize()
+    assert np.array_equal(outs2[0].float().cpu().numpy(), res["out"]) and np.array_equal(outs2[1].float().cpu().numpy(), res["out_sp"])
+    with pytest.raises(NotImplementedError):
+        ba.exact_attn(batch["q"][0], batch["kb"][0], batch["vb"][0])
+
+
+def test_k8_bad_indices_and_pages_are_skipped_and_tails_may_hold_anything(oracle_mod):
+    """The 8-bit calls treat host-made faults like the 16-bit ones: an out-of-range index or page id sets a status bit and the
+    key takes no part in the softmax; value rows and key codes beyond the prefix are NaN patterns here."""
+    o = oracle_mod
+    w = W.Workload("bad8", H_q=8, H_kv=2, N=640, B=32, k=64, T=2, n_heavy=16, page_size=64, seed=2)
+    batch = W.make_batch(w, device="cuda", steps=2)
+    n = 600                                                                  # not a multiple of 64: a ragged last tile
+    batch["seq_lens"] = torch.tensor([n], dtype=torch.int32, device="cuda")
+    batch["vc"][:, :, n:] = float("nan")
+    f = lambda t: t.float().cpu().numpy()
+    Kc, Vc = f(batch["kc"][0, :, :n]), f(batch["vc"][0, :, :n])
+    for paged in (False, True):
+        res = _run(batch, w, paged, w.k)
+        kv, k8 = res["kv"], res["k8"]
+        idx = torch.from_numpy(res["idx"]).cuda()
+        keff = torch.from_numpy(res["keff"]).cuda()
+        idx[0, 0, 5] = 1 << 28
+        idx[0, 1, 0] = -7
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        out = torch.full((kv.P, kv.H_q, kv.B, kv.d), float("nan"), dtype=torch.bfloat16, device="cuda")
+        mb.mage_sparse_block_attn_k8(kv, k8, batch["q"][1], batch["kb"][1], batch["vb"][1], idx, keff, w.k, kv.d ** -0.5, out, kv.new_workspace(w.k), status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == mb.DEV_BAD_INDEX
+        idx_left = np.stack([np.delete(res["idx"][0, 0], 5), np.delete(res["idx"][0, 1], 0)])
+        Qc1, Kcc, Kbc1, s_q1, s_k = o.k8_quantize_block(f(batch["q"][1, 0]), Kc, f(batch["kb"][1, 0]))
+        O = o.k8_sparse_block_attn(Qc1, Kcc, Vc, Kbc1, f(batch["vb"][1, 0]), idx_left, w.k - 1, s_q1, s_k)
+        err = np.abs(out.float().cpu().numpy()[0] - O)
+        assert err.max() <= H.O_MAX_ABS and err.mean() <= H.O_MEAN_ABS, (paged, err.max(), err.mean())
+    # a page id out of range in Step 1 (paged run above): its 64 keys are skipped by the attention and get score 0
+    res["table"][0, 3] = 10 ** 6
+    status.zero_()
+    scores = torch.full((kv.P, kv.H_kv, kv.N_max), -1.0, dtype=torch.float32, device="cuda")
+    mb.mage_exact_select_k8(kv, k8, batch["q"][0], batch["kb"][0], batch["vb"][0], kv.d ** -0.5, out, scores, kv.new_workspace(w.k), status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == mb.DEV_BAD_PAGE
+    keep = np.r_[0:192, 256:n]
+    Qc, Kcc, Kbc, s_q, s_k = o.k8_quantize_block(f(batch["q"][0, 0]), Kc, f(batch["kb"][0, 0]))   # scales from the whole prefix, as the GPU's
+    O = o.k8_exact_block_attn(Qc, Kcc[:, keep], Vc[:, keep], Kbc, f(batch["vb"][0, 0]), s_q, s_k)
+    err = np.abs(out.float().cpu().numpy()[0] - O)
+    assert err.max() <= H.O_MAX_ABS and err.mean() <= H.O_MEAN_ABS, (err.max(), err.mean())
+    sc = o.k8_block_score(Qc, Kcc[:, keep], s_q, s_k)
+    got = scores.cpu().numpy()[0].astype(np.float64)
+    assert (got[:, 192:256] == 0.0).all() and (got[:, n:] == -1.0).all()
+    assert np.max(np.abs(got[:, keep] - sc) / sc) <= H.SCORE_REL
