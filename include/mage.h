@@ -314,7 +314,8 @@ mage_status mage_quest_select(const mage_kv_t *kv, const void *q, const void *pa
  *   Contiguous caches need strides that are multiples of 16 elements.
  * mage_exact_select_k8 / mage_sparse_block_attn_k8 are mage_exact_select / mage_sparse_block_attn with the keys taken from
  * the codes: kv->k_cache is not read (it may be NULL); kv->v_cache, q, k_blk, v_blk, the outputs and the workspace are as
- * there.  Each call first codes its queries and block keys into k8->scratch (one small kernel).
+ * there.  The queries and block keys of a call are coded on the way: by one small kernel in front, into k8->scratch, for
+ * Step 1 and for a reuse step with more than 256 query rows per KV head; inside the kernel for the other reuse steps.
  *   k8->scratch  device, 256-byte aligned, at least mage_k8_scratch_bytes(kv); contents are per call
  * Not available with MAGE_FLAG_SIMT_KERNELS, and the reuse step needs a cache that is one list of rows with a single pitch
  * (every paged pool; contiguous layouts whose head and problem strides are multiples of the row stride): otherwise

@@ -299,7 +299,13 @@ static mage_status launch_sparse_step(const mage_kv_t *kv, const KvView &view, c
     const void *q_src = k8 ? (const void *)k8->q8 : (const void *)q, *kc_src = k8 ? (const void *)k8->k8 : kv->k_cache;
     const void *kb_src = k8 ? (const void *)k8->kb8 : (const void *)k_blk;
     if (!tc::make_group_rows_map(&maps.q, q_src, heads, view.M, eb)) return MAGE_ERR_UNSUPPORTED;
+    // 8-bit keys with one row group per head: the kernel codes the queries and the block's keys itself (no kernel in front)
+    const bool k8_fused = k8 && view.M <= 256;
     if (k8) maps.qk_scale = k8->qk_scale;
+    if (k8_fused) {
+        maps.q_raw = q;
+        maps.k_scale = k8->k_scale;
+    }
     maps.k = maps.v = maps.kb = maps.vb = maps.q;         // placeholders unless the TMA row gather below applies
     // Two gathers inside the one kernel: single 256-byte rows by TMA when the cache is one list of rows with a single pitch
     // (every paged pool; contiguous layouts whose head and problem strides are multiples of the row stride), otherwise
@@ -338,7 +344,7 @@ static mage_status launch_sparse_step(const mage_kv_t *kv, const KvView &view, c
         if (n_split > plan.sparse_split_max) n_split = plan.sparse_split_max;
         if (n_split < 1) n_split = 1;
     }
-    if (k8 && launch_block_codes(view, *k8, q, k_blk, st) != MAGE_OK) return MAGE_ERR_CUDA;
+    if (k8 && !k8_fused && launch_block_codes(view, *k8, q, k_blk, st) != MAGE_OK) return MAGE_ERR_CUDA;
     launch_pdl(kern_tc, dim3(n_split, n_rg, heads), dim3(tc::kSparseThreads), tc::kAttnSmemBytesSparse, st, maps, view, plan, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, ws, out, dev_status);
     if (launch_check() != MAGE_OK) return MAGE_ERR_CUDA;
     if (n_split > 1) {

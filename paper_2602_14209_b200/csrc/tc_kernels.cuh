@@ -8,6 +8,7 @@
 #include <type_traits>
 #include "common.cuh"
 #include "sm100_ptx.cuh"
+#include "k8.cuh"
 
 namespace mage {
 namespace tc {
@@ -462,6 +463,10 @@ struct AttnMaps {
     int rowsum_tiles = 0;
     int test_stall = 0;          // MAGE_FLAG_TEST_STALL: the exact pass never requests its first key tile and waits with the short limit
     const float *qk_scale = nullptr;   // 8-bit keys: s_q s_k per (problem, KV head); q, k, kb are then maps of e4m3 codes
+    // 8-bit keys, reuse step with at most 256 query rows per KV head: the kernel codes the queries and the block's keys
+    // itself (no kernel in front of it, no q / kb maps): the bf16 queries, and the key scale of each (problem, KV head)
+    const __nv_bfloat16 *q_raw = nullptr;
+    const float *k_scale = nullptr;
 };
 
 // K8: queries and keys (cache and block) are e4m3 codes in rows of 128 bytes; a Q or K tile then fills the first d-"half"
@@ -483,7 +488,8 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
     constexpr int kAttnSlots = SPARSE ? kAttnSlotsSparse : kAttnSlotsDense;
     const int chunk = blockIdx.x, rg = blockIdx.y, z = blockIdx.z, p = z / kv.H_kv, h = z % kv.H_kv;
     const int N = seq_len_of(kv, p);
-    if (K8) scale_log2 *= maps.qk_scale[z];
+    const bool fused_codes = K8 && SPARSE && maps.q_raw != nullptr;
+    if (K8 && !fused_codes) scale_log2 *= maps.qk_scale[z];
     int n_keys, n_cache, j_begin = 0, first_idx = 0;
     bool blk_chunk = false;
     if (!SPARSE) {
@@ -561,12 +567,33 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
         fence_mbar_init();
         fence_proxy_async();
         // the queries start their way in at once: (d, row within the KV head's G*B rows, head); rows past the head read as zeros
-        mbar_arrive_expect_tx(bar(Q_FULL), n_mt * (K8 ? kHalfBytes : kTileBytes));
-        for (int mt = 0; mt < n_mt; ++mt)
-            for (int dh = 0; dh < (K8 ? 1 : 2); ++dh)
-                for (int rb = 0; rb < 2; ++rb)
-                    tma_load_3d(smem_u32(q_s + mt * kTileBytes + dh * kHalfBytes + rb * kBoxBytes), &maps.q, bar(Q_FULL), dh * 64,
-                                rg * 256 + mt * kTile + rb * 64, z);
+        if (!fused_codes) {
+            mbar_arrive_expect_tx(bar(Q_FULL), n_mt * (K8 ? kHalfBytes : kTileBytes));
+            for (int mt = 0; mt < n_mt; ++mt)
+                for (int dh = 0; dh < (K8 ? 1 : 2); ++dh)
+                    for (int rb = 0; rb < 2; ++rb)
+                        tma_load_3d(smem_u32(q_s + mt * kTileBytes + dh * kHalfBytes + rb * kBoxBytes), &maps.q, bar(Q_FULL), dh * 64,
+                                    rg * 256 + mt * kTile + rb * 64, z);
+        }
+    }
+    // 8-bit keys, coded here: every thread fetches its share of the head's bf16 queries (all G*B <= 256 rows: one row group)
+    // and of the block's keys now, so that the loads run under the set-up and the index look-ups below.
+    uint4 fq[8], fb[2];
+    uint8_t *kb_stage = q_s + kHalfBytes;                 // [B][128] codes of the block's keys (the Q tile of M-tile 0 ends at 16 KB)
+    if (K8 && SPARSE && fused_codes) {
+        const uint4 *qv = reinterpret_cast<const uint4 *>(maps.q_raw + ((size_t)(p * kv.H_q + h * kv.G) * kv.B) * kD);
+        const int n_q16 = kv.M * 8;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int j = tid + u * (int)blockDim.x;
+            const bool in = j < n_q16;
+            fq[2 * u] = in ? qv[2 * j] : make_uint4(0, 0, 0, 0);
+            fq[2 * u + 1] = in ? qv[2 * j + 1] : make_uint4(0, 0, 0, 0);
+        }
+        const uint4 *bv = reinterpret_cast<const uint4 *>(k_blk + (size_t)z * kv.B * kD);
+        const bool in = tid < kv.B * 8;
+        fb[0] = in ? bv[2 * tid] : make_uint4(0, 0, 0, 0);
+        fb[1] = in ? bv[2 * tid + 1] : make_uint4(0, 0, 0, 0);
     }
     if (warp == kMmaWarp) { tmem_alloc(smem_u32(tmem_ptr_s), 512); tmem_relinquish(); }
     // SPARSE: resolve every selected index to a cache row once (shared by the K and V gathers): bounds check,
@@ -590,9 +617,40 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             if (o < 0) my_bad = 1;
         }
     }
+    if (K8 && SPARSE && fused_codes) {
+        // s_q = amax / 448 over the head's query rows, as the kernel in front of the other 8-bit calls takes it: the same
+        // numbers in the same arithmetic, so the codes are the same bytes
+        float *red = reinterpret_cast<float *>(kb_stage + 64 * 128);
+        float m = 0.f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) m = k8::amax8(fq[u], m);
+#pragma unroll
+        for (int w = 16; w; w >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, w));
+        if (lane == 0) red[warp] = m;
+        __syncthreads();
+        m = 0.f;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) m = fmaxf(m, red[w]);
+        const float s_q = k8::scale_of(m), s_k = maps.k_scale[z];
+        scale_log2 *= s_q * s_k;
+        // Q codes into the 128-byte-swizzled tile (row r of M-tile mt at r * 128, 16-byte piece c at (c ^ (r & 7)) * 16); rows
+        // beyond the head's last query row are zero, as the tensor map's fill would leave them
+        const int n_q16 = kv.M * 8, n_all = n_mt * kTile * 8;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int j = tid + u * (int)blockDim.x;
+            if (j < n_all) {
+                const int R = j >> 3, c = j & 7, mt_ = R >> 7, r = R & 127;
+                const uint4 code = j < n_q16 ? k8::code16(fq[2 * u], fq[2 * u + 1], s_q) : make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4 *>(q_s + mt_ * kTileBytes + r * 128 + ((c ^ (r & 7)) << 4)) = code;
+            }
+        }
+        if (tid < kv.B * 8) *reinterpret_cast<uint4 *>(kb_stage + tid * 16) = k8::code16(fb[0], fb[1], s_k);
+        fence_proxy_async();                               // the tensor pipe reads the Q tile through the async proxy
+    }
     tc_fence_before_sync();
     const int any_bad = __syncthreads_or(my_bad);
     tc_fence_after_sync();
+    if (K8 && SPARSE && fused_codes && tid == 0) mbar_arrive(bar(Q_FULL));     // the Q tile is in place (no copy to wait for)
     if (threadIdx.x == 0) MAGE_STAMP(2);
     const uint32_t tmem_base = *tmem_ptr_s;
 
@@ -693,6 +751,49 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                     const bool one_piece = K8 && !is_v;
                     const int n_req = ((i == n_tiles - 1 ? last_cols : kTile) >> 2) * (one_piece ? 1 : 2);
                     const int mine = n_req > pw ? (n_req - pw + kSparseProducerWarps - 1) / kSparseProducerWarps : 0;
+                    if (K8 && fused_codes && !is_v) {
+                        // Keys coded in this kernel: cache rows come by TMA as above; the block's rows are copied from the staged
+                        // codes with plain stores (swizzled by hand), rows past the list are zero.  A lane first writes what it
+                        // copies itself and makes it visible to the tensor pipe, then the warp announces exactly the bytes its TMA
+                        // requests will bring, then those are issued.
+                        const int o = lane * kSparseProducerWarps + pw, r_in_tile = o * 4, t0 = i * kTile + r_in_tile;
+                        const int n_c = lane < mine ? min(4, max(0, n_cache - t0)) : 0;     // rows of the group that are cache rows
+                        uint8_t *dst_g = kv_s + slot * kTileBytes + r_in_tile * 128;
+                        int rows[4];
+                        if (lane < mine) {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const int t = t0 + e, r = r_in_tile + e;
+                                if (e < n_c) {
+                                    const int ro = use_tab ? row_tab[t] : resolve(t);
+                                    rows[e] = ro >= 0 ? ro : maps.gather_rows;          // beyond the tensor: zero fill
+                                } else {
+                                    const uint4 *src = reinterpret_cast<const uint4 *>(kb_stage + (t - blk_shift) * 128);
+#pragma unroll
+                                    for (int c = 0; c < 8; ++c)
+                                        *reinterpret_cast<uint4 *>(dst_g + e * 128 + ((c ^ (r & 7)) << 4)) = t < n_keys ? src[c] : make_uint4(0, 0, 0, 0);
+                                }
+                            }
+                            if (n_c < 4) fence_proxy_async();
+                        }
+                        const int tx = __reduce_add_sync(0xffffffffu, n_c * 128);
+                        __syncwarp();                          // the lanes' stores and fences come before the warp's arrival
+                        if (lane == 0) {
+                            if (tx > 0) mbar_arrive_expect_tx(bar(FULL + slot), tx);
+                            else mbar_arrive(bar(FULL + slot));
+                        }
+                        __syncwarp();
+                        if (n_c == 4) {
+                            tma_gather4_2d(smem_u32(dst_g), &maps.k, bar(FULL + slot), 0, rows[0], rows[1], rows[2], rows[3]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                if (e < n_c) tma_load_2d(smem_u32(dst_g + e * 128), &maps.k, bar(FULL + slot), 0, rows[e]);
+                        }
+                        if (tid == 256) MAGE_STAMP(40 + L);
+                        issued = L + 1;
+                        continue;
+                    }
                     if (lane == 0) {
                         if (mine > 0) mbar_arrive_expect_tx(bar(FULL + slot), mine * 512);
                         else mbar_arrive(bar(FULL + slot));

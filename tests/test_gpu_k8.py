@@ -103,6 +103,7 @@ CASES = [
     ("one_mtile", 8, 2, 1024, 32, 2, 0, 128),                   # G*B = 128: tile-parity mode, whole tiles only
     ("short_prefix", 4, 1, 90, 16, 1, 0, 128),                  # N < one tile and k > N
     ("rows_48", 6, 2, 700, 16, 3, 200, 64),                     # G*B = 48: a partly filled M-tile
+    ("rows_448", 14, 2, 900, 64, 1, 0, 128),                    # G*B = 448: two row groups (queries coded by the kernel in front)
 ]
 
 
