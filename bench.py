@@ -466,8 +466,12 @@ def main():
                 t16.append(timed(s16, False, 1)); t8.append(timed(s8, False, 1))
             stages["exact_select_ms_alternating"], stages["k8_exact_select_ms_alternating"] = sorted(t16)[2], sorted(t8)[2]
             s16(); tk(); torch.cuda.synchronize()
-            idx16 = ba.indices.clone()
+            idx16, out16 = ba.indices.clone(), outs[0].float()
             s8(); tk(); torch.cuda.synchronize()
+            diff = (outs[0].float() - out16).abs()
+            stages["k8_step1_output_vs_16bit_max_abs"], stages["k8_step1_output_vs_16bit_mean_abs"] = float(diff.max()), float(diff.mean())
+            stages["k8_step1_output_rms_16bit"] = float(out16.pow(2).mean().sqrt())
+            del out16, diff
             same = 0
             for p_ in range(kv.P):
                 for h_ in range(kv.H_kv):
