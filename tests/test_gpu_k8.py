@@ -283,3 +283,16 @@ def test_k8_bad_indices_and_pages_are_skipped_and_tails_may_hold_anything(oracle
     got = scores.cpu().numpy()[0].astype(np.float64)
     assert (got[:, 192:256] == 0.0).all() and (got[:, n:] == -1.0).all()
     assert np.max(np.abs(got[:, keep] - sc) / sc) <= H.SCORE_REL
+
+
+def test_k8_zero_queries_and_zero_keys(oracle_mod):
+    """amax = 0 takes scale 1 on both sides: an all-zero query head gives uniform attention, an all-zero key head too."""
+    w = W.Workload("zeros", H_q=8, H_kv=2, N=300, B=32, k=64, T=2, P=1, n_heavy=16, seed=17)
+    batch = W.make_batch(w, device="cuda", steps=2)
+    batch["q"][:, :, :4] = 0                      # the four query heads of KV head 0, both steps
+    batch["kc"][:, 1] = 0                         # every cached key of KV head 1
+    res = _run(batch, w, False, w.k)
+    assert res["k_scale"][0, 1] == 1.0
+    _check(oracle_mod, batch, w, res, w.k)
+    # uniform over the prefix for head 0: every score is 1 / N
+    assert np.allclose(res["scores"][0, 0, :300], 1.0 / 300, rtol=1e-5)
