@@ -334,15 +334,27 @@ static mage_status launch_sparse_step(const mage_kv_t *kv, const KvView &view, c
         if ((last >> 3) > 0x7fffffffLL) return MAGE_ERR_UNSUPPORTED;
     }
     if (opt_in_smem(kern_tc, tc::kAttnSmemBytesSparse) != MAGE_OK) return MAGE_ERR_CUDA;
-    const int n_rg = (view.M + 255) / 256;
+    int n_rg = (view.M + 255) / 256;
     // few (head, row-group) pairs in the launch: split each head's keys over several CTAs and merge
     int n_split = 1;
     if (ws_ok && plan.sparse_split_max > 1) {
-        n_split = 148 / (heads * n_rg);
         const int tiles = (k + kv->B + 127) / 128;
-        if (n_split > tiles) n_split = tiles;
-        if (n_split > plan.sparse_split_max) n_split = plan.sparse_split_max;
-        if (n_split < 1) n_split = 1;
+        auto splits_for = [&](int groups) {
+            int s = 148 / (heads * groups);
+            if (s > tiles) s = tiles;
+            if (s > plan.sparse_split_max) s = plan.sparse_split_max;
+            return s < 1 ? 1 : s;
+        };
+        n_split = splits_for(n_rg);
+        // A split CTA spends most of its time writing its partial result (fp32, 512 bytes per query row); with row groups of
+        // 128 instead of 256 rows each CTA writes half of it.  Every key tile is then gathered by two CTAs, which costs more
+        // than it saves once the launch fills more than about half of the SMs (measured: 12.9 -> 11.4 us with 40 CTAs,
+        // 15.8 -> 17.3 us with 136).
+        const int n_rg128 = (view.M + 127) / 128;
+        if (n_split > 1 && n_rg128 > n_rg && !k8_fused && splits_for(n_rg128) == n_split && heads * n_rg128 * n_split <= 74) {
+            n_rg = n_rg128;
+            maps.rg_rows = 128;
+        }
     }
     if (k8 && !k8_fused && launch_block_codes(view, *k8, q, k_blk, st) != MAGE_OK) return MAGE_ERR_CUDA;
     launch_pdl(kern_tc, dim3(n_split, n_rg, heads), dim3(tc::kSparseThreads), tc::kAttnSmemBytesSparse, st, maps, view, plan, k_blk, v_blk, indices, k_eff, k, sm_scale * kLog2e, ws, out, dev_status);

@@ -467,6 +467,9 @@ struct AttnMaps {
     // itself (no kernel in front of it, no q / kb maps): the bf16 queries, and the key scale of each (problem, KV head)
     const __nv_bfloat16 *q_raw = nullptr;
     const float *k_scale = nullptr;
+    // query rows per CTA (blockIdx.y counts groups of this many rows of a KV head): 256, or 128 for a reuse step that is split
+    // over CTAs anyway -- a 128-row CTA writes half the partial result, which is most of what such a CTA spends its time on
+    int rg_rows = 256;
 };
 
 // K8: queries and keys (cache and block) are e4m3 codes in rows of 128 bytes; a Q or K tile then fills the first d-"half"
@@ -525,7 +528,8 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
     // Reuse step: the last tile of the list usually holds little more than the block's own keys; it is gathered, multiplied
     // and exponentiated at its own width (a multiple of 16 keys) instead of a full 128.
     const int last_cols = SPARSE ? ((n_keys - (n_tiles - 1) * kTile + 15) & ~15) : kTile;
-    const int rows_here = min(256, kv.M - rg * 256), n_mt = rows_here > 128 ? 2 : 1;
+    const int rgr = SPARSE ? maps.rg_rows : 256;         // query rows per row group
+    const int rows_here = min(rgr, kv.M - rg * rgr), n_mt = rows_here > 128 ? 2 : 1;
     // With a single M-tile the second softmax warpgroup and the second S/O regions would idle.  They take the
     // odd key tiles instead ("tile-parity mode"): two independent online-softmax pipelines over the same 128 rows,
     // each with its own reference, sum and O accumulator, merged by warpgroup 0 at the end.
@@ -573,7 +577,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 for (int dh = 0; dh < (K8 ? 1 : 2); ++dh)
                     for (int rb = 0; rb < 2; ++rb)
                         tma_load_3d(smem_u32(q_s + mt * kTileBytes + dh * kHalfBytes + rb * kBoxBytes), &maps.q, bar(Q_FULL), dh * 64,
-                                    rg * 256 + mt * kTile + rb * 64, z);
+                                    rg * rgr + mt * kTile + rb * 64, z);
         }
     }
     // 8-bit keys, coded here: every thread fetches its share of the head's bf16 queries (all G*B <= 256 rows: one row group)
@@ -1042,8 +1046,8 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
             const uint32_t lane_off = (uint32_t)(w4 * 32) << 16;
             const uint32_t tS = tmem_base + mt * 128 + lane_off, tO = tmem_base + 256 + mt * 128 + lane_off;
             const int first = tp ? mt : 0, stride = tp ? 2 : 1;      // tiles of this warpgroup: first, first + stride, ...
-            const int row = w4 * 32 + lane, grow = rg * 256 + (tp ? 0 : mt * kTile) + row;
-            const bool warp_has_rows = rg * 256 + (tp ? 0 : mt * kTile) + w4 * 32 < kv.M;
+            const int row = w4 * 32 + lane, grow = rg * rgr + (tp ? 0 : mt * kTile) + row;
+            const bool warp_has_rows = rg * rgr + (tp ? 0 : mt * kTile) + w4 * 32 < kv.M;
             float m_used = -INFINITY, l = 0.f;
             float pend_m = 0.f;          // reference the row wants to move to at the start of its next tile
             bool pending = false;
@@ -1345,7 +1349,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, KvView kv, Plan plan, const _
                 // whole 256-byte pieces, two rows per instruction.
                 constexpr int kStageRow = 256 + 16;
                 uint8_t *stg = kv_s + warp * (32 * kStageRow);
-                const int row0 = rg * 256 + (tp ? 0 : mt * kTile) + w4 * 32;              // first row of this warp
+                const int row0 = rg * rgr + (tp ? 0 : mt * kTile) + w4 * 32;              // first row of this warp
                 const int rows_ok = min(32, kv.M - row0);                                   // may be <= 0
                 auto flush = [&](uint8_t *dst_row0, size_t dst_pitch) {                     // 32 staged rows of 256 bytes -> global
                     __syncwarp();
